@@ -1,0 +1,154 @@
+/*
+ * slide_attn.h -- C ABI of the fused Slide Attention forward for NVIDIA B200 (sm_100a).
+ *
+ * The operation (Slide-Transformer, arXiv 2304.04237):
+ *
+ *   For every query pixel p = (b, i, j) of a [B, H, W] map and every head h:
+ *
+ *     Ks[s, c] = sum_t wk[c, s, t] * K0(p + off(t), c)        Sec. 4.2, Eq. 12: depthwise k x k
+ *     Vs[s, c] = sum_t wv[c, s, t] * V0(p + off(t), c)        convolution per slot s; wk / wv are
+ *                                                             the merged kernels of Sec. 4.3
+ *                                                             (fixed shift, Eq. 11, + learned
+ *                                                             deformed shift, re-parameterised)
+ *     l[s]     = (sum_{c in head h} q[p, c] * Ks[s, c]) / sqrt(head_dim)  (+ bias[h, s])    Eq. 2
+ *     a        = softmax over the k*k slots of l                                            Eq. 2
+ *     out[p,c] = sum_s a[s] * Vs[s, c]                                                      Eq. 2
+ *
+ *   r = floor(k/2); slot s = (u+r)*k + (v+r) for the window offset (u, v) in [-r, r]^2
+ *   (Eq. 4-9, row-major over (u, v)); tap t = p_*k + q_ for the kernel position (p_, q_) in
+ *   [0, k)^2 with off(t) = (p_ - r, q_ - r) (Eq. 12; cross-correlation, no kernel flip).
+ *   K0 / V0 read zero outside the map ("[1,1] padding", Fig. 2); padded slots are NOT masked:
+ *   they take part in the softmax with key 0 and value 0, as a zero-padded convolution gives.
+ *   With wk = wv = the one-hot kernels (w[c, s, t] = 1 iff t == s) the result is plain k x k
+ *   local attention (Sec. 3.2 (3)).
+ *
+ * The k*k-expanded keys and values are never written to device memory: convolution, logits,
+ * softmax and aggregation run in one kernel.
+ *
+ * Tensor layouts (all dense, row-major, no strides):
+ *   q, k, v, out : [B][H][W][heads][head_dim], element type = the context's dtype
+ *                  (channel c = h*head_dim + e; "channels-last")
+ *   wk, wv       : float [C][k*k slot][k*k tap], C = heads*head_dim.  This is the memory of a
+ *                  PyTorch-style depthwise weight [C*k*k, 1, k, k] with groups = C and output
+ *                  channel c*k*k + s, so a re-parameterised convolution weight can be passed as is.
+ *   bias         : float [heads][k*k], or NULL
+ *
+ * Ownership: the caller owns every tensor.  The library reads/writes them only in stream order
+ * within the call that received them and keeps no pointer afterwards.  A context owns a small
+ * device workspace (re-laid-out weights, a status word), allocated by slide_attn_create.
+ *
+ * Errors: every function returns a status code; nothing is thrown or printed; no device code
+ * traps.  Arguments are validated on the host before anything is launched.  There is no CPU
+ * fallback: on a device that is not sm_100 slide_attn_create returns SLIDE_ATTN_ERR_ARCH.
+ *
+ * Threading: one context must not be used from two host threads at once, and two forwards on
+ * the same context must be ordered on the device (same stream, or events), because they share
+ * the context's workspace.  Distinct contexts are independent.
+ */
+#ifndef SLIDE_ATTN_H_
+#define SLIDE_ATTN_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct slide_attn_ctx slide_attn_ctx;      /* opaque; created and destroyed by the library */
+
+typedef enum {
+    SLIDE_ATTN_F32  = 0,    /* q, k, v, out are IEEE float                                        */
+    SLIDE_ATTN_BF16 = 1     /* q, k, v, out are bfloat16; arithmetic accumulates in float         */
+} slide_attn_dtype;
+
+typedef enum {
+    SLIDE_ATTN_OK = 0,
+    SLIDE_ATTN_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, unknown enum             */
+    SLIDE_ATTN_ERR_UNSUPPORTED = 2,   /* even ksize, ksize > 15, head_dim not a multiple of 8, ...  */
+    SLIDE_ATTN_ERR_ALIGNMENT   = 3,   /* a tensor pointer is not 16-byte aligned                   */
+    SLIDE_ATTN_ERR_ALLOC       = 4,   /* device or host allocation failed                          */
+    SLIDE_ATTN_ERR_CUDA        = 5,   /* a CUDA runtime/driver call failed                         */
+    SLIDE_ATTN_ERR_ARCH        = 6,   /* current device is not compute capability 10.x             */
+    SLIDE_ATTN_ERR_TIMEOUT     = 7    /* a bounded device-side wait ran out (see query_status)     */
+} slide_attn_status;
+
+/* Kernel variants.  AUTO picks the fastest one that supports the context's shape; the others
+ * exist for A/B measurements and tests.  All variants compute the same function. */
+typedef enum {
+    SLIDE_ATTN_VARIANT_AUTO    = 0,
+    SLIDE_ATTN_VARIANT_DIRECT  = 1,   /* one warp per (pixel, head), global loads, fp32 FMA; any shape */
+    SLIDE_ATTN_VARIANT_TILED   = 2,   /* halo tile in shared memory, fp32 FMA on CUDA cores            */
+    SLIDE_ATTN_VARIANT_MMA     = 3    /* halo tile in shared memory, deformed-shift contraction on
+                                         tensor cores (bf16 operands, fp32 accumulate); bf16 only       */
+} slide_attn_variant;
+
+/*
+ * Creates a context for one problem shape on the CURRENT CUDA device (Eq. 2 over a k x k window;
+ * shapes as in the layout section above).
+ *   ctx       [out, host]  receives the context; untouched on error
+ *   B, H, W   batch and map size, each >= 1 (H or W smaller than ksize is legal)
+ *   heads, head_dim        >= 1; head_dim must be a multiple of 8 and <= 256
+ *   ksize     odd, 1..15 (the window offsets u, v range over [-floor(k/2), floor(k/2)], which
+ *             is centred only for odd k)
+ *   dtype     element type of q, k, v, out
+ *   has_bias  non-zero if forward will be given a bias
+ * Allocates the context's workspace (cudaMalloc); synchronous.
+ */
+slide_attn_status slide_attn_create(slide_attn_ctx** ctx,
+                                    int B, int H, int W, int heads, int head_dim, int ksize,
+                                    slide_attn_dtype dtype, int has_bias);
+
+/*
+ * Runs the forward (the five formulas at the top; Eq. 2, Eq. 12, Sec. 4.3) asynchronously on
+ * `cuda_stream` (a cudaStream_t; NULL = the legacy default stream).
+ *   q, k, v   [in,  DEVICE] [B][H][W][heads][head_dim], ctx dtype, 16-byte aligned
+ *   wk, wv    [in,  DEVICE] float [C][k*k][k*k], 16-byte aligned
+ *   bias      [in,  DEVICE] float [heads][k*k]; must be non-NULL iff the context has_bias
+ *   out       [out, DEVICE] same shape and dtype as q, 16-byte aligned; must not alias an input
+ * Does not allocate and does not synchronise; the result is deterministic (bit-identical from
+ * run to run for a given variant).  Weight re-layout, where a variant needs it, happens inside
+ * this call on the same stream, so wk / wv may change between calls.
+ */
+slide_attn_status slide_attn_forward(slide_attn_ctx* ctx,
+                                     const void* q, const void* k, const void* v,
+                                     const float* wk, const float* wv, const float* bias,
+                                     void* out, void* cuda_stream);
+
+/*
+ * The same forward (Eq. 2, Eq. 12, Sec. 4.3) for HOST buffers of the same layouts: copies q, k,
+ * v, wk, wv, bias to device staging buffers owned by the context, runs slide_attn_forward,
+ * copies `out` back and waits for the stream.  Page-locked host buffers make the copies
+ * asynchronous with respect to other streams; pageable ones work too.  The staging buffers are
+ * allocated on the first call (cudaMalloc) and reused afterwards.
+ */
+slide_attn_status slide_attn_forward_host(slide_attn_ctx* ctx,
+                                          const void* q, const void* k, const void* v,
+                                          const float* wk, const float* wv, const float* bias,
+                                          void* out, void* cuda_stream);
+
+/* Selects the kernel variant used by later forwards.  SLIDE_ATTN_ERR_UNSUPPORTED if the variant
+ * cannot run the context's shape or dtype (the previous choice stays). */
+slide_attn_status slide_attn_set_variant(slide_attn_ctx* ctx, slide_attn_variant variant);
+
+/* The variant the next forward will run (never AUTO).  *variant [out, host]. */
+slide_attn_status slide_attn_get_variant(const slide_attn_ctx* ctx, slide_attn_variant* variant);
+
+/* Number of kernels one slide_attn_forward launches with the current variant.  *n [out, host]. */
+slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* ctx, int* n);
+
+/*
+ * Waits for `cuda_stream` and reports the device-side status word: SLIDE_ATTN_OK, or
+ * SLIDE_ATTN_ERR_TIMEOUT if a kernel gave up on a bounded wait (its output is then undefined).
+ * The word is cleared by this call.
+ */
+slide_attn_status slide_attn_query_status(slide_attn_ctx* ctx, void* cuda_stream);
+
+/* Frees the context and everything it owns.  NULL is accepted.  The caller must make sure no
+ * forward of this context is still running. */
+slide_attn_status slide_attn_destroy(slide_attn_ctx* ctx);
+
+/* A static, NUL-terminated description of a status code. */
+const char* slide_attn_status_string(slide_attn_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SLIDE_ATTN_H_ */

@@ -1,0 +1,38 @@
+// Shared declarations of the slide-attention library: problem description, element access,
+// and the launchers each kernel file exports to the API layer.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "slide_attn.h"
+
+namespace slide_attn {
+
+// One forward problem.  Channel c = h*head_dim + e; C = heads*head_dim; k2 = ksize*ksize.
+struct Problem {
+    int B, H, W, heads, head_dim, ksize;
+    int has_bias;
+    slide_attn_dtype dtype;
+    const void* q;
+    const void* k;
+    const void* v;
+    const float* wk;     // [C][k2 slot][k2 tap]
+    const float* wv;
+    const float* bias;   // [heads][k2] or nullptr
+    void* out;
+};
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_float(float x);
+template <> __device__ __forceinline__ float from_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float x) {
+    return __float2bfloat16_rn(x);
+}
+
+// Launchers.  Each returns cudaGetLastError() of its launch(es).
+cudaError_t launch_direct(const Problem& p, cudaStream_t stream);
+bool direct_supports(int head_dim, int ksize);
+
+}  // namespace slide_attn

@@ -1,0 +1,237 @@
+// C-ABI layer of the slide-attention library: argument validation, the context, variant
+// selection and the host-buffer entry point.  All arithmetic lives in the kernel files.
+#include <new>
+
+#include "common.cuh"
+
+using namespace slide_attn;
+
+struct slide_attn_ctx {
+    int B, H, W, heads, head_dim, ksize, has_bias;
+    slide_attn_dtype dtype;
+    slide_attn_variant variant;      // never AUTO
+    int device;
+    int* d_status;                   // device status word (0 = ok)
+    void* workspace;                 // re-laid-out weights for the variants that need them
+    size_t workspace_bytes;
+    // staging buffers for slide_attn_forward_host, allocated on first use
+    void* stage;
+    size_t stage_bytes;
+};
+
+namespace {
+
+size_t elem_size(slide_attn_dtype t) { return t == SLIDE_ATTN_BF16 ? 2 : 4; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
+    switch (v) {
+        case SLIDE_ATTN_VARIANT_DIRECT: return direct_supports(c->head_dim, c->ksize);
+        default: return false;
+    }
+}
+
+slide_attn_variant pick_variant(const slide_attn_ctx* c) {
+    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_TILED,
+                                        SLIDE_ATTN_VARIANT_DIRECT};
+    for (slide_attn_variant v : order)
+        if (variant_supported(c, v)) return v;
+    return SLIDE_ATTN_VARIANT_DIRECT;
+}
+
+slide_attn_status validate_shape(int B, int H, int W, int heads, int head_dim, int ksize,
+                                 slide_attn_dtype dtype) {
+    if (B < 1 || H < 1 || W < 1 || heads < 1 || head_dim < 1 || ksize < 1)
+        return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (dtype != SLIDE_ATTN_F32 && dtype != SLIDE_ATTN_BF16) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if ((ksize & 1) == 0 || ksize > 15) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    if (head_dim % 8 != 0 || head_dim > 256) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    // element counts must fit the kernels' index arithmetic
+    const long long n = (long long)B * H * W;
+    if (n > (1LL << 40) / ((long long)heads * head_dim)) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    return SLIDE_ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, int heads,
+                                    int head_dim, int ksize, slide_attn_dtype dtype, int has_bias)
+{
+    if (!ctx) return SLIDE_ATTN_ERR_INVALID_ARG;
+    slide_attn_status st = validate_shape(B, H, W, heads, head_dim, ksize, dtype);
+    if (st != SLIDE_ATTN_OK) return st;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    if (major != 10) return SLIDE_ATTN_ERR_ARCH;
+
+    slide_attn_ctx* c = new (std::nothrow) slide_attn_ctx();
+    if (!c) return SLIDE_ATTN_ERR_ALLOC;
+    c->B = B; c->H = H; c->W = W; c->heads = heads; c->head_dim = head_dim; c->ksize = ksize;
+    c->has_bias = has_bias ? 1 : 0;
+    c->dtype = dtype;
+    c->device = dev;
+    c->d_status = nullptr; c->workspace = nullptr; c->workspace_bytes = 0;
+    c->stage = nullptr; c->stage_bytes = 0;
+    if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess ||
+        cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        slide_attn_destroy(c);
+        return SLIDE_ATTN_ERR_ALLOC;
+    }
+    c->variant = pick_variant(c);
+    *ctx = c;
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_forward(slide_attn_ctx* c, const void* q, const void* k, const void* v,
+                                     const float* wk, const float* wv, const float* bias,
+                                     void* out, void* cuda_stream)
+{
+    if (!c || !q || !k || !v || !wk || !wv || !out) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if ((c->has_bias != 0) != (bias != nullptr)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (out == q || out == k || out == v) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(wk) ||
+        !aligned16(wv) || (bias && !aligned16(bias)))
+        return SLIDE_ATTN_ERR_ALIGNMENT;
+
+    Problem p;
+    p.B = c->B; p.H = c->H; p.W = c->W; p.heads = c->heads; p.head_dim = c->head_dim;
+    p.ksize = c->ksize; p.has_bias = c->has_bias; p.dtype = c->dtype;
+    p.q = q; p.k = k; p.v = v; p.wk = wk; p.wv = wv; p.bias = bias; p.out = out;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    cudaError_t err;
+    switch (c->variant) {
+        case SLIDE_ATTN_VARIANT_DIRECT: err = launch_direct(p, stream); break;
+        default: return SLIDE_ATTN_ERR_UNSUPPORTED;
+    }
+    return err == cudaSuccess ? SLIDE_ATTN_OK : SLIDE_ATTN_ERR_CUDA;
+}
+
+slide_attn_status slide_attn_forward_host(slide_attn_ctx* c, const void* q, const void* k,
+                                          const void* v, const float* wk, const float* wv,
+                                          const float* bias, void* out, void* cuda_stream)
+{
+    if (!c || !q || !k || !v || !wk || !wv || !out) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if ((c->has_bias != 0) != (bias != nullptr)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const size_t C = (size_t)c->heads * c->head_dim, k2 = (size_t)c->ksize * c->ksize;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t t_raw = (size_t)c->B * c->H * c->W * C * elem_size(c->dtype);
+    const size_t w_raw = C * k2 * k2 * sizeof(float);
+    const size_t b_raw = (size_t)c->heads * k2 * sizeof(float);
+    const size_t t_bytes = up(t_raw), w_bytes = up(w_raw), b_bytes = up(b_raw);
+    const size_t total = 4 * t_bytes + 2 * w_bytes + b_bytes;
+    if (c->stage_bytes < total) {
+        if (c->stage) { cudaFree(c->stage); c->stage = nullptr; c->stage_bytes = 0; }
+        if (cudaMalloc(&c->stage, total) != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_ALLOC; }
+        c->stage_bytes = total;
+    }
+    char* base = static_cast<char*>(c->stage);
+    void* dq = base;
+    void* dk = base + t_bytes;
+    void* dv = base + 2 * t_bytes;
+    void* dout = base + 3 * t_bytes;
+    float* dwk = reinterpret_cast<float*>(base + 4 * t_bytes);
+    float* dwv = reinterpret_cast<float*>(base + 4 * t_bytes + w_bytes);
+    float* dbias = reinterpret_cast<float*>(base + 4 * t_bytes + 2 * w_bytes);
+
+    bool ok = cudaMemcpyAsync(dq, q, t_raw, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dk, k, t_raw, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dv, v, t_raw, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dwk, wk, w_raw, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dwv, wv, w_raw, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (ok && bias)
+        ok = cudaMemcpyAsync(dbias, bias, b_raw, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+
+    slide_attn_status st = slide_attn_forward(c, dq, dk, dv, dwk, dwv, bias ? dbias : nullptr, dout, stream);
+    if (st != SLIDE_ATTN_OK) return st;
+    if (cudaMemcpyAsync(out, dout, t_raw, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant variant)
+{
+    if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (variant == SLIDE_ATTN_VARIANT_AUTO) { c->variant = pick_variant(c); return SLIDE_ATTN_OK; }
+    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_MMA)
+        return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!variant_supported(c, variant)) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    c->variant = variant;
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_get_variant(const slide_attn_ctx* c, slide_attn_variant* variant)
+{
+    if (!c || !variant) return SLIDE_ATTN_ERR_INVALID_ARG;
+    *variant = c->variant;
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* n)
+{
+    if (!c || !n) return SLIDE_ATTN_ERR_INVALID_ARG;
+    switch (c->variant) {
+        case SLIDE_ATTN_VARIANT_DIRECT: *n = 1; break;
+        default: *n = 1; break;
+    }
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_query_status(slide_attn_ctx* c, void* cuda_stream)
+{
+    if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemsetAsync(c->d_status, 0, sizeof(int), stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    return word == 0 ? SLIDE_ATTN_OK : SLIDE_ATTN_ERR_TIMEOUT;
+}
+
+slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
+{
+    if (!c) return SLIDE_ATTN_OK;
+    bool ok = true;
+    if (c->d_status) ok &= cudaFree(c->d_status) == cudaSuccess;
+    if (c->workspace) ok &= cudaFree(c->workspace) == cudaSuccess;
+    if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
+    delete c;
+    if (!ok) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+    return SLIDE_ATTN_OK;
+}
+
+const char* slide_attn_status_string(slide_attn_status status)
+{
+    switch (status) {
+        case SLIDE_ATTN_OK: return "ok";
+        case SLIDE_ATTN_ERR_INVALID_ARG: return "invalid argument";
+        case SLIDE_ATTN_ERR_UNSUPPORTED: return "unsupported shape, window size or variant";
+        case SLIDE_ATTN_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case SLIDE_ATTN_ERR_ALLOC: return "allocation failed";
+        case SLIDE_ATTN_ERR_CUDA: return "CUDA call failed";
+        case SLIDE_ATTN_ERR_ARCH: return "device is not sm_100 (B200)";
+        case SLIDE_ATTN_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,332 @@
+"""Benchmark of the fused Slide Attention forward.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--variant auto]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores, same metric
+
+One step = one forward of the whole hot path (depthwise shift/deform convolution of K and V,
+logits, softmax, aggregation) over one batch of seeded synthetic feature maps.  Prints ONE JSON
+line (rank 0).  With N > 1 (torchrun) every rank runs the full batch on its own GPU: the batch
+axis shards with no exchange, so there is no collective on the data path ("weak" scaling).
+
+Timing: CUDA events on the launching stream around exactly K steps, barrier + synchronize on both
+sides, max over ranks.  Inputs rotate over several buffer sets whose total size exceeds twice the
+L2 capacity, so every step reads its inputs from HBM.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2304_04237_b200 import synth  # noqa: E402
+
+METRIC = "slide_attn_fwd_query_pixels_per_s"
+UNIT = "query-pixels/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def algorithmic_bytes(cfg) -> int:
+    """Minimal HBM traffic of one forward: q, k, v read once, out written once, fp32 weights
+    of both convolutions and the bias read once."""
+    n = cfg["B"] * cfg["H"] * cfg["W"]
+    C = cfg["heads"] * cfg["head_dim"]
+    k2 = cfg["ksize"] ** 2
+    sz = 2 if cfg["dtype"] == "bf16" else 4
+    return n * C * 4 * sz + 2 * C * k2 * k2 * 4 + (cfg["heads"] * k2 * 4 if cfg["has_bias"] else 0)
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {"sm_mhz": (float(np.median(self.samples)) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def cpu_oracle_rate(cfg, x, budget_s=15.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: whole images
+    taken from the front of the batch.  Returns (pixels/s, threads, description)."""
+    import oracle
+    hw = cfg["H"] * cfg["W"]
+    nb = min(2, x["q"].shape[0])
+    args = lambda n: (x["q"][:n], x["k"][:n], x["v"][:n], x["wk"], x["wv"], x["bias"], cfg["ksize"])
+    t0 = time.perf_counter()
+    oracle.forward(*args(nb))
+    probe = time.perf_counter() - t0
+    n_img = int(max(1, min(x["q"].shape[0], budget_s / max(probe / nb, 1e-9))))
+    t0 = time.perf_counter()
+    oracle.forward(*args(n_img))
+    dt = time.perf_counter() - t0
+    return n_img * hw / dt, oracle.threads(), f"first {n_img} of {cfg['B']} images of the workload ({n_img * hw} query pixels, {dt:.1f} s)"
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores; rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = dict(synth.CONFIGS[args.workload])
+    # inputs for as many images as one step's sample may need
+    x = synth.make_inputs(batch_limit=min(cfg["B"], 16), **cfg)
+    import oracle
+    hw = cfg["H"] * cfg["W"]
+    t0 = time.perf_counter()
+    oracle.forward(x["q"][:1], x["k"][:1], x["v"][:1], x["wk"], x["wv"], x["bias"], cfg["ksize"])
+    per_img = time.perf_counter() - t0
+    total_steps = args.steps + args.warmup
+    n_img = int(max(1, min(x["q"].shape[0], 60.0 / total_steps / max(per_img, 1e-9))))
+    call = lambda: oracle.forward(x["q"][:n_img], x["k"][:n_img], x["v"][:n_img], x["wk"], x["wv"],
+                                  x["bias"], cfg["ksize"])
+    for _ in range(args.warmup):
+        call()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        call()
+    dt = time.perf_counter() - t0
+    value = args.steps * n_img * hw / dt
+    sample = f"each step = first {n_img} of {cfg['B']} images ({n_img * hw} query pixels)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(cfg, args.workload, None),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, name, l2_note):
+    c = {"workload": f"{name}: B={cfg['B']} H={cfg['H']} W={cfg['W']} heads={cfg['heads']} "
+                     f"head_dim={cfg['head_dim']} k={cfg['ksize']} {cfg['dtype']} "
+                     f"bias={'yes' if cfg['has_bias'] else 'no'} sigma_w={cfg['sigma_w']}",
+         "name": name, "B": cfg["B"], "H": cfg["H"], "W": cfg["W"], "heads": cfg["heads"],
+         "head_dim": cfg["head_dim"], "ksize": cfg["ksize"], "storage_dtype": cfg["dtype"]}
+    if l2_note:
+        c["l2"] = l2_note
+    return c
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--variant", default="auto", choices=["auto", "direct", "tiled", "mma"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2304_04237_b200 as sa
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = dict(synth.CONFIGS[args.workload])
+    x = synth.make_inputs(**cfg)
+    td = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
+    host = {n: torch.from_numpy(x[n]).to(td) for n in ("q", "k", "v")}
+    wk, wv = torch.from_numpy(x["wk"]).cuda(), torch.from_numpy(x["wv"]).cuda()
+    bias = None if x["bias"] is None else torch.from_numpy(x["bias"]).cuda()
+
+    # rotating buffer sets: total > 2 x L2 so that no step finds its inputs in cache
+    l2 = torch.cuda.get_device_properties(local).L2_cache_size
+    set_bytes = 4 * host["q"].numel() * host["q"].element_size()
+    n_sets = max(2, int(np.ceil(2.0 * l2 / set_bytes)) + 1)
+    sets = []
+    for i in range(n_sets):
+        s = {n: host[n].cuda() for n in ("q", "k", "v")}
+        s["out"] = torch.empty_like(s["q"])
+        sets.append(s)
+    l2_note = (f"{n_sets} rotating (q,k,v,out) buffer sets, {n_sets * set_bytes / 1e6:.0f} MB in total "
+               f"> 2 x L2 ({l2 / 1e6:.0f} MB)")
+
+    ctx = sa.slide_attn_create(cfg["B"], cfg["H"], cfg["W"], cfg["heads"], cfg["head_dim"],
+                               cfg["ksize"], td, cfg["has_bias"])
+    if args.variant != "auto":
+        sa.slide_attn_set_variant(ctx, {"direct": 1, "tiled": 2, "mma": 3}[args.variant])
+    variant = {1: "direct", 2: "tiled", 3: "mma"}[sa.slide_attn_get_variant(ctx)]
+    launches = sa.slide_attn_launches_per_forward(ctx)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        s = sets[i % n_sets]
+        sa.slide_attn_forward(ctx, s["q"], s["k"], s["v"], wk, wv, bias, s["out"], stream)
+
+    def fence():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    fence()
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    sa.slide_attn_profile_begin(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    fence()
+    clocks = sampler.stop()
+    fwd_ms, main_ms, n_prof = sa.slide_attn_profile_end(ctx)
+    assert sa.slide_attn_query_status(ctx) == sa.OK
+    total_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    npx = cfg["B"] * cfg["H"] * cfg["W"]
+    value = world * npx / (ms_per_step * 1e-3)
+
+    # end to end through the host-buffer entry point: pinned host inputs in, pinned result out
+    e2e = None
+    if args.e2e_steps > 0:
+        pin = {n: host[n].pin_memory() for n in ("q", "k", "v")}
+        pwk, pwv = torch.from_numpy(x["wk"]).pin_memory(), torch.from_numpy(x["wv"]).pin_memory()
+        pb = None if x["bias"] is None else torch.from_numpy(x["bias"]).pin_memory()
+        pout = torch.empty_like(pin["q"]).pin_memory()
+        for _ in range(2):
+            sa.slide_attn_forward_host(ctx, pin["q"], pin["k"], pin["v"], pwk, pwv, pb, pout, stream)
+        fence()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            sa.slide_attn_forward_host(ctx, pin["q"], pin["k"], pin["v"], pwk, pwv, pb, pout, stream)
+        b.record(stream)
+        fence()
+        e2e_ms = a.elapsed_time(b) / args.e2e_steps
+        if world > 1:
+            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        h2d = 3 * pin["q"].numel() * pin["q"].element_size() + 2 * pwk.numel() * 4 + (0 if pb is None else pb.numel() * 4)
+        e2e = {"value": world * npx / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(pout.numel() * pout.element_size()),
+               "steps": args.e2e_steps}
+    sa.slide_attn_destroy(ctx)
+
+    if rank == 0:
+        peak, peak_src = hbm_peak()
+        abytes = algorithmic_bytes(cfg)
+        achieved = abytes / (main_ms * 1e-3) / 1e9 if main_ms > 0 else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if cfg["dtype"] == "f32" else "bf16 storage, f32 accumulate",
+            "data": "synthetic", "config": workload_config(cfg, args.workload, l2_note),
+            "variant": variant, "gpu_launches": launches * args.steps,
+            "hbm_gbs_algorithmic": abytes / (ms_per_step * 1e-3) / 1e9,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": (achieved / peak if achieved else None), "traffic": None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": abytes,
+                         "kernel_ms": main_ms, "forward_ms": fwd_ms, "launches_averaged": n_prof},
+            "clocks": clocks, "e2e": e2e,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            v, cores, sample = cpu_oracle_rate(cfg, x)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": sample}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -141,6 +141,19 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* ctx, int
  */
 slide_attn_status slide_attn_query_status(slide_attn_ctx* ctx, void* cuda_stream);
 
+/*
+ * Kernel timing for benchmarks (no counterpart in the paper's text; it measures the fused kernel
+ * of Eq. 2 / Eq. 12).  After slide_attn_profile_begin every slide_attn_forward on this context
+ * records CUDA events on its stream around (a) all kernels of the call and (b) the main fused
+ * kernel alone; up to 1024 forwards are kept (later ones overwrite the oldest).
+ * slide_attn_profile_end waits for the recorded events and reports the mean durations in
+ * milliseconds and the number of forwards averaged, then stops recording.
+ *   forward_ms, main_ms, n  [out, host]; any may be NULL.
+ * Events cost a few microseconds of host time per forward; leave profiling off otherwise.
+ */
+slide_attn_status slide_attn_profile_begin(slide_attn_ctx* ctx);
+slide_attn_status slide_attn_profile_end(slide_attn_ctx* ctx, double* forward_ms, double* main_ms, int* n);
+
 /* Frees the context and everything it owns.  NULL is accepted.  The caller must make sure no
  * forward of this context is still running. */
 slide_attn_status slide_attn_destroy(slide_attn_ctx* ctx);

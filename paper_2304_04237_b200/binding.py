@@ -20,6 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALLOC, ERR_CUDA, ERR_AR
 
 EXPORTS = ("slide_attn_create", "slide_attn_forward", "slide_attn_forward_host",
            "slide_attn_set_variant", "slide_attn_get_variant", "slide_attn_launches_per_forward",
+           "slide_attn_profile_begin", "slide_attn_profile_end",
            "slide_attn_query_status", "slide_attn_destroy", "slide_attn_status_string")
 
 _lib = None
@@ -47,6 +48,9 @@ def load() -> ctypes.CDLL:
         lib.slide_attn_set_variant.argtypes = [vp, i]
         lib.slide_attn_get_variant.argtypes = [vp, ctypes.POINTER(i)]
         lib.slide_attn_launches_per_forward.argtypes = [vp, ctypes.POINTER(i)]
+        lib.slide_attn_profile_begin.argtypes = [vp]
+        lib.slide_attn_profile_end.argtypes = [vp, ctypes.POINTER(ctypes.c_double),
+                                               ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i)]
         lib.slide_attn_query_status.argtypes = [vp, vp]
         lib.slide_attn_destroy.argtypes = [vp]
         lib.slide_attn_status_string.argtypes = [i]
@@ -125,6 +129,18 @@ def slide_attn_launches_per_forward(ctx) -> int:
     n = ctypes.c_int()
     _check(load().slide_attn_launches_per_forward(ctx, ctypes.byref(n)), "slide_attn_launches_per_forward")
     return n.value
+
+
+def slide_attn_profile_begin(ctx) -> None:
+    _check(load().slide_attn_profile_begin(ctx), "slide_attn_profile_begin")
+
+
+def slide_attn_profile_end(ctx):
+    """Returns (mean ms per forward, mean ms of the main kernel, forwards averaged)."""
+    f, m, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
+    _check(load().slide_attn_profile_end(ctx, ctypes.byref(f), ctypes.byref(m), ctypes.byref(n)),
+           "slide_attn_profile_end")
+    return f.value, m.value, n.value
 
 
 def slide_attn_query_status(ctx, stream=None) -> int:

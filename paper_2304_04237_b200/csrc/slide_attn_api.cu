@@ -17,9 +17,15 @@ struct slide_attn_ctx {
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
     size_t stage_bytes;
+    // profiling: ring of event triples (start, before main kernel, end)
+    bool profiling;
+    int prof_count;                  // forwards recorded since profile_begin
+    cudaEvent_t* prof_events;        // kProfRing * 3, created on the first profile_begin
 };
 
 namespace {
+
+constexpr int kProfRing = 1024;
 
 size_t elem_size(slide_attn_dtype t) { return t == SLIDE_ATTN_BF16 ? 2 : 4; }
 
@@ -81,6 +87,7 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
     c->device = dev;
     c->d_status = nullptr; c->workspace = nullptr; c->workspace_bytes = 0;
     c->stage = nullptr; c->stage_bytes = 0;
+    c->profiling = false; c->prof_count = 0; c->prof_events = nullptr;
     if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess ||
         cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) {
         cudaGetLastError();
@@ -109,10 +116,22 @@ slide_attn_status slide_attn_forward(slide_attn_ctx* c, const void* q, const voi
     p.q = q; p.k = k; p.v = v; p.wk = wk; p.wv = wv; p.bias = bias; p.out = out;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
+    cudaEvent_t* ev = nullptr;
+    if (c->profiling) {
+        ev = c->prof_events + 3 * (c->prof_count % kProfRing);
+        cudaEventRecord(ev[0], stream);
+    }
     cudaError_t err;
     switch (c->variant) {
-        case SLIDE_ATTN_VARIANT_DIRECT: err = launch_direct(p, stream); break;
+        case SLIDE_ATTN_VARIANT_DIRECT:
+            if (ev) cudaEventRecord(ev[1], stream);
+            err = launch_direct(p, stream);
+            break;
         default: return SLIDE_ATTN_ERR_UNSUPPORTED;
+    }
+    if (ev) {
+        cudaEventRecord(ev[2], stream);
+        c->prof_count++;
     }
     return err == cudaSuccess ? SLIDE_ATTN_OK : SLIDE_ATTN_ERR_CUDA;
 }
@@ -193,6 +212,51 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
     return SLIDE_ATTN_OK;
 }
 
+slide_attn_status slide_attn_profile_begin(slide_attn_ctx* c)
+{
+    if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!c->prof_events) {
+        cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[3 * kProfRing];
+        if (!ev) return SLIDE_ATTN_ERR_ALLOC;
+        for (int i = 0; i < 3 * kProfRing; ++i) {
+            if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+                cudaGetLastError();
+                for (int j = 0; j < i; ++j) cudaEventDestroy(ev[j]);
+                delete[] ev;
+                return SLIDE_ATTN_ERR_CUDA;
+            }
+        }
+        c->prof_events = ev;
+    }
+    c->prof_count = 0;
+    c->profiling = true;
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_profile_end(slide_attn_ctx* c, double* forward_ms, double* main_ms, int* n)
+{
+    if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!c->profiling) return SLIDE_ATTN_ERR_INVALID_ARG;
+    c->profiling = false;
+    const int cnt = c->prof_count < kProfRing ? c->prof_count : kProfRing;
+    double fwd = 0.0, mn = 0.0;
+    for (int i = 0; i < cnt; ++i) {
+        cudaEvent_t* ev = c->prof_events + 3 * i;
+        float a = 0.f, b = 0.f;
+        if (cudaEventSynchronize(ev[2]) != cudaSuccess ||
+            cudaEventElapsedTime(&a, ev[0], ev[2]) != cudaSuccess ||
+            cudaEventElapsedTime(&b, ev[1], ev[2]) != cudaSuccess) {
+            cudaGetLastError();
+            return SLIDE_ATTN_ERR_CUDA;
+        }
+        fwd += a; mn += b;
+    }
+    if (forward_ms) *forward_ms = cnt ? fwd / cnt : 0.0;
+    if (main_ms) *main_ms = cnt ? mn / cnt : 0.0;
+    if (n) *n = cnt;
+    return SLIDE_ATTN_OK;
+}
+
 slide_attn_status slide_attn_query_status(slide_attn_ctx* c, void* cuda_stream)
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
@@ -214,6 +278,10 @@ slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
     if (c->d_status) ok &= cudaFree(c->d_status) == cudaSuccess;
     if (c->workspace) ok &= cudaFree(c->workspace) == cudaSuccess;
     if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
+    if (c->prof_events) {
+        for (int i = 0; i < 3 * kProfRing; ++i) ok &= cudaEventDestroy(c->prof_events[i]) == cudaSuccess;
+        delete[] c->prof_events;
+    }
     delete c;
     if (!ok) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
     return SLIDE_ATTN_OK;

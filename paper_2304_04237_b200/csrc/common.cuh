@@ -35,4 +35,13 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(f
 cudaError_t launch_direct(const Problem& p, cudaStream_t stream);
 bool direct_supports(int head_dim, int ksize);
 
+// MMA variant.  `workspace` holds the re-laid-out weights (mma_workspace_bytes), written by the
+// prep launch and read by the main launch on the same stream.  mma_setup must have succeeded once
+// on the device before the first main launch.
+bool mma_supports(slide_attn_dtype dtype, int head_dim, int ksize);
+size_t mma_workspace_bytes(int heads);
+cudaError_t mma_setup();
+cudaError_t launch_mma_prep(const Problem& p, void* workspace, cudaStream_t stream);
+cudaError_t launch_mma_main(const Problem& p, const void* workspace, int* d_status, cudaStream_t stream);
+
 }  // namespace slide_attn

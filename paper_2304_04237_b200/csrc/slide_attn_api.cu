@@ -34,6 +34,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
     switch (v) {
         case SLIDE_ATTN_VARIANT_DIRECT: return direct_supports(c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_MMA: return c->workspace && mma_supports(c->dtype, c->head_dim, c->ksize);
         default: return false;
     }
 }
@@ -94,6 +95,20 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
         slide_attn_destroy(c);
         return SLIDE_ATTN_ERR_ALLOC;
     }
+    if (mma_supports(dtype, head_dim, ksize)) {
+        if (mma_setup() != cudaSuccess) {
+            cudaGetLastError();
+            slide_attn_destroy(c);
+            return SLIDE_ATTN_ERR_CUDA;
+        }
+        c->workspace_bytes = mma_workspace_bytes(heads);
+        if (cudaMalloc(&c->workspace, c->workspace_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            c->workspace = nullptr;
+            slide_attn_destroy(c);
+            return SLIDE_ATTN_ERR_ALLOC;
+        }
+    }
     c->variant = pick_variant(c);
     *ctx = c;
     return SLIDE_ATTN_OK;
@@ -126,6 +141,11 @@ slide_attn_status slide_attn_forward(slide_attn_ctx* c, const void* q, const voi
         case SLIDE_ATTN_VARIANT_DIRECT:
             if (ev) cudaEventRecord(ev[1], stream);
             err = launch_direct(p, stream);
+            break;
+        case SLIDE_ATTN_VARIANT_MMA:
+            err = launch_mma_prep(p, c->workspace, stream);
+            if (ev) cudaEventRecord(ev[1], stream);
+            if (err == cudaSuccess) err = launch_mma_main(p, c->workspace, c->d_status, stream);
             break;
         default: return SLIDE_ATTN_ERR_UNSUPPORTED;
     }
@@ -207,6 +227,7 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
     if (!c || !n) return SLIDE_ATTN_ERR_INVALID_ARG;
     switch (c->variant) {
         case SLIDE_ATTN_VARIANT_DIRECT: *n = 1; break;
+        case SLIDE_ATTN_VARIANT_MMA: *n = 2; break;      // weight re-layout + fused kernel
         default: *n = 1; break;
     }
     return SLIDE_ATTN_OK;

@@ -189,8 +189,8 @@ def workload_config(cfg, name, l2_note):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
     ap.add_argument("--variant", default="auto", choices=["auto", "direct", "tiled", "mma"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

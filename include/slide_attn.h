@@ -67,7 +67,8 @@ typedef enum {
     SLIDE_ATTN_ERR_ALLOC       = 4,   /* device or host allocation failed                          */
     SLIDE_ATTN_ERR_CUDA        = 5,   /* a CUDA runtime/driver call failed                         */
     SLIDE_ATTN_ERR_ARCH        = 6,   /* current device is not compute capability 10.x             */
-    SLIDE_ATTN_ERR_TIMEOUT     = 7    /* a bounded device-side wait ran out (see query_status)     */
+    SLIDE_ATTN_ERR_TIMEOUT     = 7,   /* a bounded device-side wait ran out (see query_status)     */
+    SLIDE_ATTN_ERR_TOO_LARGE   = 8    /* problem exceeds the fixed scratch of forward_noalloc      */
 } slide_attn_status;
 
 /* Kernel variants.  AUTO picks the fastest one that supports the context's shape; the others
@@ -140,6 +141,40 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* ctx, int
  * The word is cleared by this call.
  */
 slide_attn_status slide_attn_query_status(slide_attn_ctx* ctx, void* cuda_stream);
+
+/*
+ * Forward without a context and without any allocation.  (The paper has no counterpart to this
+ * entry point; it computes the same Eq. 2 / Eq. 12 forward as slide_attn_forward.)
+ *
+ * Who needs it: callers that are not allowed to allocate device memory -- code that runs inside a
+ * memory plan with fixed buffers (an inference engine's arena, a plugin), a process whose
+ * allocator is frozen after start-up, or a latency-critical loop that cannot afford the implicit
+ * device synchronisation of cudaMalloc / cudaFree.  slide_attn_create allocates, so such callers
+ * cannot use a context.  Here the scratch memory of the tensor-core variant (re-laid-out weights,
+ * status word) is a fixed array inside the library's device image instead; every GPU that loads
+ * the library holds it (288.25 KiB) until the process exits.  This call performs no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ * Arguments: tensors as for slide_attn_forward (DEVICE pointers, same layouts, 16-byte aligned,
+ * bias may be NULL), followed by the shape the context would have carried.
+ * Limits: dtype SLIDE_ATTN_BF16, head_dim 32, ksize 3 (else SLIDE_ATTN_ERR_UNSUPPORTED);
+ * heads <= 16 (else SLIDE_ATTN_ERR_TOO_LARGE -- the fixed scratch has room for 16 heads).
+ *
+ * First call on a device: resolves the scratch's device address and configures the kernel
+ * (no allocation, but driver calls that are not legal during stream capture) -- make the first
+ * call on each device outside of any stream capture, with that device current.
+ *
+ * Sharing: every call on a device uses the same scratch, and the scratch keeps the previous call's
+ * contents.  Each call rewrites all of it that it reads and clears the status word first, so
+ * back-to-back calls on ONE stream are safe; calls that may overlap on the GPU (different streams
+ * without an event between them, or several host threads) race on the scratch and give undefined
+ * results.  Device-side time-outs are not reported by this entry point.
+ */
+slide_attn_status slide_attn_forward_noalloc(const void* q, const void* k, const void* v,
+                                             const float* wk, const float* wv, const float* bias,
+                                             void* out,
+                                             int B, int H, int W, int heads, int head_dim, int ksize,
+                                             slide_attn_dtype dtype, void* cuda_stream);
 
 /*
  * Kernel timing for benchmarks (no counterpart in the paper's text; it measures the fused kernel

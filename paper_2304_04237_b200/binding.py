@@ -17,8 +17,10 @@ LIB_PATH = os.path.join(_HERE, "libslide_attn.so")
 F32, BF16 = 0, 1
 VARIANT_AUTO, VARIANT_DIRECT, VARIANT_TILED, VARIANT_MMA = 0, 1, 2, 3
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(8)
+ERR_TOO_LARGE = 8
 
 EXPORTS = ("slide_attn_create", "slide_attn_forward", "slide_attn_forward_host",
+           "slide_attn_forward_noalloc",
            "slide_attn_set_variant", "slide_attn_get_variant", "slide_attn_launches_per_forward",
            "slide_attn_profile_begin", "slide_attn_profile_end",
            "slide_attn_query_status", "slide_attn_destroy", "slide_attn_status_string")
@@ -45,6 +47,7 @@ def load() -> ctypes.CDLL:
         lib.slide_attn_create.argtypes = [ctypes.POINTER(vp), i, i, i, i, i, i, i, i]
         lib.slide_attn_forward.argtypes = [vp] * 9
         lib.slide_attn_forward_host.argtypes = [vp] * 9
+        lib.slide_attn_forward_noalloc.argtypes = [vp] * 7 + [i] * 7 + [vp]
         lib.slide_attn_set_variant.argtypes = [vp, i]
         lib.slide_attn_get_variant.argtypes = [vp, ctypes.POINTER(i)]
         lib.slide_attn_launches_per_forward.argtypes = [vp, ctypes.POINTER(i)]
@@ -113,6 +116,18 @@ def slide_attn_forward_host(ctx, q, k, v, wk, wv, bias, out, stream=None) -> Non
     """CPU tensors in and out (pinned for best speed); returns when `out` is filled."""
     _check(load().slide_attn_forward_host(ctx, *map(_host_ptr, (q, k, v, wk, wv, bias, out)),
                                           _stream_ptr(stream)), "slide_attn_forward_host")
+
+
+def slide_attn_forward_noalloc(q, k, v, wk, wv, bias, out, ksize, stream=None) -> None:
+    """Forward for callers that must not allocate device memory: no context, the library's
+    fixed scratch is used instead (bf16, head_dim 32, ksize 3, at most 16 heads).  The shape is
+    taken from `q` ([B, H, W, heads, head_dim]).  Calls that overlap on the GPU race on the
+    shared scratch; keep them on one stream."""
+    B, H, W, heads, head_dim = q.shape
+    dtype = {torch.float32: F32, torch.bfloat16: BF16}[q.dtype]
+    _check(load().slide_attn_forward_noalloc(*map(_dev_ptr, (q, k, v, wk, wv, bias, out)),
+                                             B, H, W, heads, head_dim, int(ksize), dtype,
+                                             _stream_ptr(stream)), "slide_attn_forward_noalloc")
 
 
 def slide_attn_set_variant(ctx, variant: int) -> None:

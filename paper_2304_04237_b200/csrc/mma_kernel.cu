@@ -20,6 +20,8 @@
 // 8*tig .. 8*tig+7, i.e. rows g and g+8 of two 16-row MMA tiles (rows 0,1 and rows 2,3).
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace slide_attn {
@@ -460,3 +462,104 @@ cudaError_t launch_mma_main(const Problem& p, const void* workspace, int* d_stat
 }
 
 }  // namespace slide_attn
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free entry point.
+//
+// Some callers may not allocate device memory at all: code running inside a memory-planned
+// region (a framework's static arena, a plugin that is handed fixed buffers), a process whose
+// allocator is locked down after start-up, or a latency-critical loop where cudaMalloc's implicit
+// device synchronisation is not acceptable.  slide_attn_create allocates, so those callers cannot
+// hold a context.  For them the scratch of the MMA variant (the re-laid-out weights and the
+// status word) lives in the fixed arrays below, which every GPU that loads this library keeps
+// until the process exits: kStaticMaxHeads * 18 432 B + 256 B = 288.25 KiB.
+// ---------------------------------------------------------------------------------------------
+namespace slide_attn {
+namespace {
+
+constexpr int kStaticMaxHeads = 16;
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) uint32_t g_static_frag[kStaticMaxHeads * kFragWordsPerHead];
+static __device__ __align__(256) int g_static_status[64];
+
+// In host code the two names above are host-side stand-ins, not device addresses; the addresses
+// the kernels get are resolved per device with cudaGetSymbolAddress.
+struct StaticScratch {
+    bool ready;
+    uint32_t* frag;
+    int* status;
+};
+StaticScratch g_scratch[kStaticMaxDevices];
+std::mutex g_scratch_mutex;
+
+slide_attn_status static_scratch(int dev, StaticScratch* out) {
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    StaticScratch& s = g_scratch[dev];
+    if (!s.ready) {
+        if (mma_setup() != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+        void* frag = nullptr;
+        void* status = nullptr;
+        if (cudaGetSymbolAddress(&frag, g_static_frag) != cudaSuccess ||
+            cudaGetSymbolAddress(&status, g_static_status) != cudaSuccess || !frag || !status) {
+            cudaGetLastError();
+            return SLIDE_ATTN_ERR_CUDA;
+        }
+        s.frag = static_cast<uint32_t*>(frag);
+        s.status = static_cast<int*>(status);
+        s.ready = true;
+    }
+    *out = s;
+    return SLIDE_ATTN_OK;
+}
+
+}  // namespace
+}  // namespace slide_attn
+
+extern "C" slide_attn_status slide_attn_forward_noalloc(
+    const void* q, const void* k, const void* v, const float* wk, const float* wv, const float* bias,
+    void* out, int B, int H, int W, int heads, int head_dim, int ksize, slide_attn_dtype dtype,
+    void* cuda_stream)
+{
+    using namespace slide_attn;
+    if (!q || !k || !v || !wk || !wv || !out) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (B < 1 || H < 1 || W < 1 || heads < 1 || head_dim < 1 || ksize < 1) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (dtype != SLIDE_ATTN_F32 && dtype != SLIDE_ATTN_BF16) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (out == q || out == k || out == v) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!mma_supports(dtype, head_dim, ksize)) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    if (heads > kStaticMaxHeads) return SLIDE_ATTN_ERR_TOO_LARGE;
+    if ((long long)B * H * W > (1LL << 40) / ((long long)heads * head_dim)) return SLIDE_ATTN_ERR_TOO_LARGE;
+    auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out) || misaligned(wk) ||
+        misaligned(wv) || (bias && misaligned(bias)))
+        return SLIDE_ATTN_ERR_ALIGNMENT;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+    if (dev < 0 || dev >= kStaticMaxDevices) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    if (major != 10) return SLIDE_ATTN_ERR_ARCH;
+
+    StaticScratch scratch;
+    slide_attn_status st = static_scratch(dev, &scratch);
+    if (st != SLIDE_ATTN_OK) return st;
+
+    Problem p;
+    p.B = B; p.H = H; p.W = W; p.heads = heads; p.head_dim = head_dim; p.ksize = ksize;
+    p.has_bias = bias != nullptr; p.dtype = dtype;
+    p.q = q; p.k = k; p.v = v; p.wk = wk; p.wv = wv; p.bias = bias; p.out = out;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The fragment words of the heads in use are all rewritten by the prep launch; the status
+    // word is the only thing that has to start at zero.
+    if (cudaMemsetAsync(scratch.status, 0, sizeof(int), stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    cudaError_t err = launch_mma_prep(p, scratch.frag, stream);
+    if (err == cudaSuccess) err = launch_mma_main(p, scratch.frag, scratch.status, stream);
+    return err == cudaSuccess ? SLIDE_ATTN_OK : SLIDE_ATTN_ERR_CUDA;
+}

@@ -319,6 +319,7 @@ const char* slide_attn_status_string(slide_attn_status status)
         case SLIDE_ATTN_ERR_CUDA: return "CUDA call failed";
         case SLIDE_ATTN_ERR_ARCH: return "device is not sm_100 (B200)";
         case SLIDE_ATTN_ERR_TIMEOUT: return "device-side wait timed out";
+        case SLIDE_ATTN_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of slide_attn_forward_noalloc (16 heads)";
         default: return "unknown status";
     }
 }

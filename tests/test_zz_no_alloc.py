@@ -1,0 +1,74 @@
+"""The allocation-free entry point, slide_attn_forward_noalloc.
+
+It exists for callers that may not allocate device memory (fixed memory plans, frozen
+allocators, loops that cannot take cudaMalloc's synchronisation) and therefore cannot create a
+context; its scratch is a fixed array inside the library.  Checked here against the ordinary
+context-based forward on the same inputs, twice in a row with different data and head counts,
+because the scratch is shared by all calls and keeps the previous call's contents.
+
+Collected last on purpose: a run that stops at the first failure has then already run every
+other test."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2304_04237_b200 as sa
+from paper_2304_04237_b200 import synth
+
+from util import TOL, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _context_forward(dev, shape):
+    B, H, W, heads, d = shape
+    out = torch.full_like(dev["q"], float("nan"))
+    ctx = sa.slide_attn_create(B, H, W, heads, d, 3, torch.bfloat16, dev["bias"] is not None)
+    try:
+        sa.slide_attn_set_variant(ctx, sa.VARIANT_MMA)
+        sa.slide_attn_forward(ctx, dev["q"], dev["k"], dev["v"], dev["wk"], dev["wv"], dev["bias"], out)
+        torch.cuda.synchronize()
+    finally:
+        sa.slide_attn_destroy(ctx)
+    return out
+
+
+def test_noalloc_matches_context_forward_on_two_calls_in_a_row():
+    cases = [((2, 21, 30, 3, 32), True, 0.05, 11), ((1, 40, 17, 2, 32), False, 0.3, 12)]
+    prepared = []
+    for shape, has_bias, sigma_w, seed in cases:
+        B, H, W, heads, d = shape
+        x = synth.make_inputs(B, H, W, heads, d, 3, "bf16", sigma_w, 0.2, has_bias, seed=seed)
+        dev = to_device(x, "bf16")
+        prepared.append((shape, dev, _context_forward(dev, shape)))
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    outs = []
+    for shape, dev, _ in prepared:                      # two calls back to back, same stream
+        out = torch.full_like(dev["q"], float("nan"))
+        outs.append(out)
+    allocated_for_outputs = torch.cuda.memory_allocated() - before
+    for (shape, dev, _), out in zip(prepared, outs):
+        sa.slide_attn_forward_noalloc(dev["q"], dev["k"], dev["v"], dev["wk"], dev["wv"], dev["bias"], out, 3)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() - before == allocated_for_outputs
+    for (shape, dev, want), out in zip(prepared, outs):
+        got, ref = out.float().cpu().numpy().astype(np.float64), want.float().cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        err = np.abs(got - ref) / np.maximum(1.0, np.abs(ref))
+        assert err.max() <= TOL["bf16"], (shape, err.max())
+
+
+def test_noalloc_rejects_what_its_fixed_scratch_cannot_hold():
+    lib = sa.binding.load()
+    t = torch.zeros(1, 4, 8, 17, 32, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(17 * 32, 9, 9, device="cuda")
+    o = torch.empty_like(t)
+    args = lambda heads, d, k, dt: (t.data_ptr(), t.data_ptr(), t.data_ptr(), w.data_ptr(), w.data_ptr(), None,
+                                    o.data_ptr(), 1, 4, 8, heads, d, k, dt, None)
+    assert lib.slide_attn_forward_noalloc(*args(17, 32, 3, sa.BF16)) == sa.ERR_TOO_LARGE
+    assert "16 heads" in sa.slide_attn_status_string(sa.ERR_TOO_LARGE)
+    assert lib.slide_attn_forward_noalloc(*args(2, 32, 5, sa.BF16)) == sa.ERR_UNSUPPORTED
+    assert lib.slide_attn_forward_noalloc(*args(2, 64, 3, sa.BF16)) == sa.ERR_UNSUPPORTED
+    assert lib.slide_attn_forward_noalloc(*args(2, 32, 3, sa.F32)) == sa.ERR_UNSUPPORTED
+    torch.cuda.synchronize()

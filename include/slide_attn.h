@@ -76,9 +76,12 @@ typedef enum {
 typedef enum {
     SLIDE_ATTN_VARIANT_AUTO    = 0,
     SLIDE_ATTN_VARIANT_DIRECT  = 1,   /* one warp per (pixel, head), global loads, fp32 FMA; any shape */
-    SLIDE_ATTN_VARIANT_TILED   = 2,   /* halo tile in shared memory, fp32 FMA on CUDA cores            */
-    SLIDE_ATTN_VARIANT_MMA     = 3    /* halo tile in shared memory, deformed-shift contraction on
-                                         tensor cores (bf16 operands, fp32 accumulate); bf16 only       */
+    SLIDE_ATTN_VARIANT_MMA     = 2,   /* TMA halo tile in shared memory, deformed-shift contraction on
+                                         tensor cores (bf16 operands, fp32 accumulate); one CTA per
+                                         tile and head; bf16, head_dim 32, ksize 3                      */
+    SLIDE_ATTN_VARIANT_MMA_WS  = 3    /* same arithmetic, persistent warp-specialised schedule (key
+                                         warps / value warps, 3-stage TMA ring, weights resident in
+                                         registers, single launch); bf16, head_dim 32, ksize 3          */
 } slide_attn_variant;
 
 /*

@@ -44,4 +44,10 @@ cudaError_t mma_setup();
 cudaError_t launch_mma_prep(const Problem& p, void* workspace, cudaStream_t stream);
 cudaError_t launch_mma_main(const Problem& p, const void* workspace, int* d_status, cudaStream_t stream);
 
+
+// MMA_WS variant: persistent warp-specialised kernel, single launch, no workspace.
+bool mma_ws_supports(slide_attn_dtype dtype, int head_dim, int ksize);
+cudaError_t mma_ws_setup();
+cudaError_t launch_mma_ws(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
+
 }  // namespace slide_attn

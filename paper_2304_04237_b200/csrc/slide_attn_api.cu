@@ -11,6 +11,7 @@ struct slide_attn_ctx {
     slide_attn_dtype dtype;
     slide_attn_variant variant;      // never AUTO
     int device;
+    int num_sms;
     int* d_status;                   // device status word (0 = ok)
     void* workspace;                 // re-laid-out weights for the variants that need them
     size_t workspace_bytes;
@@ -35,12 +36,13 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
     switch (v) {
         case SLIDE_ATTN_VARIANT_DIRECT: return direct_supports(c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_MMA: return c->workspace && mma_supports(c->dtype, c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_MMA_WS: return mma_ws_supports(c->dtype, c->head_dim, c->ksize);
         default: return false;
     }
 }
 
 slide_attn_variant pick_variant(const slide_attn_ctx* c) {
-    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_TILED,
+    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_MMA_WS, SLIDE_ATTN_VARIANT_MMA,
                                         SLIDE_ATTN_VARIANT_DIRECT};
     for (slide_attn_variant v : order)
         if (variant_supported(c, v)) return v;
@@ -79,6 +81,11 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
         return SLIDE_ATTN_ERR_CUDA;
     }
     if (major != 10) return SLIDE_ATTN_ERR_ARCH;
+    int num_sms = 0;
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 1) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
 
     slide_attn_ctx* c = new (std::nothrow) slide_attn_ctx();
     if (!c) return SLIDE_ATTN_ERR_ALLOC;
@@ -86,6 +93,7 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
     c->has_bias = has_bias ? 1 : 0;
     c->dtype = dtype;
     c->device = dev;
+    c->num_sms = num_sms;
     c->d_status = nullptr; c->workspace = nullptr; c->workspace_bytes = 0;
     c->stage = nullptr; c->stage_bytes = 0;
     c->profiling = false; c->prof_count = 0; c->prof_events = nullptr;
@@ -96,7 +104,7 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
         return SLIDE_ATTN_ERR_ALLOC;
     }
     if (mma_supports(dtype, head_dim, ksize)) {
-        if (mma_setup() != cudaSuccess) {
+        if (mma_setup() != cudaSuccess || mma_ws_setup() != cudaSuccess) {
             cudaGetLastError();
             slide_attn_destroy(c);
             return SLIDE_ATTN_ERR_CUDA;
@@ -146,6 +154,10 @@ slide_attn_status slide_attn_forward(slide_attn_ctx* c, const void* q, const voi
             err = launch_mma_prep(p, c->workspace, stream);
             if (ev) cudaEventRecord(ev[1], stream);
             if (err == cudaSuccess) err = launch_mma_main(p, c->workspace, c->d_status, stream);
+            break;
+        case SLIDE_ATTN_VARIANT_MMA_WS:
+            if (ev) cudaEventRecord(ev[1], stream);
+            err = launch_mma_ws(p, c->d_status, c->num_sms, stream);
             break;
         default: return SLIDE_ATTN_ERR_UNSUPPORTED;
     }
@@ -208,7 +220,7 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant v
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (variant == SLIDE_ATTN_VARIANT_AUTO) { c->variant = pick_variant(c); return SLIDE_ATTN_OK; }
-    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_MMA)
+    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_MMA_WS)
         return SLIDE_ATTN_ERR_INVALID_ARG;
     if (!variant_supported(c, variant)) return SLIDE_ATTN_ERR_UNSUPPORTED;
     c->variant = variant;
@@ -228,6 +240,7 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
     switch (c->variant) {
         case SLIDE_ATTN_VARIANT_DIRECT: *n = 1; break;
         case SLIDE_ATTN_VARIANT_MMA: *n = 2; break;      // weight re-layout + fused kernel
+        case SLIDE_ATTN_VARIANT_MMA_WS: *n = 1; break;
         default: *n = 1; break;
     }
     return SLIDE_ATTN_OK;

@@ -15,7 +15,7 @@ from util import TORCH_DTYPE, VARIANTS, assert_close, gpu_forward, to_device
 
 pytestmark = pytest.mark.gpu
 
-ALL_VARIANTS = ["auto", "direct", "tiled", "mma"]
+ALL_VARIANTS = ["auto", "direct", "mma", "mma_ws"]
 
 
 def ref_forward(x, k):

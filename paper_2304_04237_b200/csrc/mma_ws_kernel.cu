@@ -4,14 +4,21 @@
 // start; Eq. 2 with Eq. 12 inside), different schedule:
 //
 //   * one CTA per SM, each bound to ONE head for its whole life, looping over 4 x TW pixel tiles;
-//   * 4 key warps and 8 value warps.  A key warp keeps all key-side B fragments (72 registers) and
+//   * key warps and value warps.  A key warp keeps all key-side B fragments (72 registers) and
 //     turns a unit (4 rows x 8 columns) into unnormalised softmax weights e[p, 0..8] and 1/sum; a
 //     value warp keeps all value-side B fragments and turns e into the output.  e travels through
-//     a small double-buffered shared-memory mailbox per value warp, guarded by mbarriers;
+//     a ring of shared-memory mailboxes (one per unit in flight), guarded by mbarriers;
 //   * K / V halo tiles and the q tile arrive by TMA (zero fill outside the map = the padding of the
 //     convolution) into a 3-stage ring; lane 0 of key warp 0 is the producer;
 //   * the fp32 weights of the head are brought in once by two 1-D bulk copies and every warp builds
 //     its own fragments from them, so there is no separate weight-prep launch and no workspace.
+//
+// Lane (g, tig) = (lane/4, lane%4) owns column g of the unit, all four rows, and channels
+// 8*tig .. 8*tig+7.  Pixel rows 2*mt and 2*mt+1 are rows g and g+8 of MMA tile mt, so the two halves
+// of an MMA read the same halo column, one row apart.  The loops walk a halo column top to bottom:
+// each halo position is loaded (and, on the value side, widened to fp32) once per lane and reused
+// by every tap that touches it.  Lanes g and g+1 read adjacent 64-byte pixels, so every 16-byte
+// shared-memory access is conflict-free without swizzling.
 //
 // Every wait is bounded; a wait that runs out sets the status word and the warp leaves.
 #include "common.cuh"
@@ -22,11 +29,12 @@ namespace slide_attn {
 namespace {
 
 constexpr int kHeadDim = 32;
-constexpr int kKWarps = 4;
-constexpr int kVWarps = 8;
+constexpr int kKWarps = 6;
+constexpr int kVWarps = 6;
 constexpr int kThreads = (kKWarps + kVWarps) * 32;
 constexpr int kMaxStages = 3;
-constexpr int kMailBytes = 8 * 10 * 4 * 4;              // [g 8][slot 0..8, 9 = 1/sum][row 4] floats
+constexpr int kMailSlots = 16;
+constexpr int kMailBytes = 8 * 10 * 4 * 4;              // [g 8][slot 0..8, 9 = 1/sum][pixel 4] floats
 constexpr int kWeightBytes = kHeadDim * 81 * 4;         // fp32 weights of one head, one side
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -44,31 +52,31 @@ struct WsParams {
 };
 
 struct Smem {
-    uint32_t halo_pad;         // bytes of one K or V halo tile (6 rows x (TW+2) pixels x 64 B), 128-aligned
-    uint32_t stage_bytes;
-    uint32_t mail_off;         // mailboxes: [value warp 8][slot 2][kMailBytes]
+    uint32_t halo_pad;         // bytes of one K or V halo tile (6 rows x (TW+2) pixels x 64 B), 1024-aligned
+    uint32_t stage_bytes;      // K halo | V halo | q tile, 1024-aligned
+    uint32_t mail_off;         // mailboxes: [kMailSlots][kMailBytes]
     uint32_t bar_off;          // mbarriers
-    uint32_t total;
+    uint32_t total;            // including 1024 bytes of slack to align the base
 };
 
 __host__ __device__ inline Smem smem_layout(int TW, int stages) {
     Smem s;
-    s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 127u) & ~127u;
-    s.stage_bytes = 2 * s.halo_pad + (uint32_t)(4 * TW * 64);
+    s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 1023u) & ~1023u;
+    s.stage_bytes = 2 * s.halo_pad + (((uint32_t)(4 * TW * 64) + 1023u) & ~1023u);
     // the last stage doubles as the staging area of the head's fp32 weights (both sides)
-    const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 127u) & ~127u;
+    const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
     if (s.stage_bytes < wbytes) s.stage_bytes = wbytes;
     s.mail_off = s.stage_bytes * stages;
-    s.bar_off = s.mail_off + kVWarps * 2 * kMailBytes;
-    s.total = s.bar_off + 64 * 8;
+    s.bar_off = s.mail_off + kMailSlots * kMailBytes;
+    s.total = s.bar_off + 64 * 8 + 1024;
     return s;
 }
 
 // barrier indices (8 bytes each) behind bar_off
-constexpr int kBarFull = 0;        // [stage]     TMA landed
-constexpr int kBarEmpty = 3;       // [stage]     all units of the tile are done with the stage
-constexpr int kBarMailFull = 6;    // [vwarp][2]  e written
-constexpr int kBarMailEmpty = 22;  // [vwarp][2]  e consumed
+constexpr int kBarFull = 0;        // [stage]  TMA landed
+constexpr int kBarEmpty = 3;       // [stage]  all units of the tile are done with the stage
+constexpr int kBarMailFull = 6;    // [slot]   e written
+constexpr int kBarMailEmpty = 22;  // [slot]   e consumed
 constexpr int kBarWeights = 38;    // weights landed
 constexpr int kBarWeightsDone = 39;  // all warps have built their fragments
 
@@ -83,7 +91,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, const WsParams P)
 {
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-aligned
     const Smem L = smem_layout(P.TW, P.stages);
     const uint32_t bar0 = smem_u32(smem + L.bar_off);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -108,7 +117,7 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             mbar_init(bar(kBarFull + s), 1);
             mbar_init(bar(kBarEmpty + s), 2 * U);
         }
-        for (int i = 0; i < 2 * kVWarps; ++i) {
+        for (int i = 0; i < kMailSlots; ++i) {
             mbar_init(bar(kBarMailFull + i), 1);
             mbar_init(bar(kBarMailEmpty + i), 1);
         }
@@ -203,7 +212,6 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
         const uint32_t ones_t1 = g == 0 ? kOnesBf16x2 : 0u;    // third n-tile: column 0 sums tap 1,
         const uint32_t ones_t8 = g == 1 ? kOnesBf16x2 : 0u;    //               column 1 sums tap 8
-        int sent0 = 0, sent1 = 0;                              // units handed to value warp `warp` / `warp + 4`
 
         for (int u = warp; ok && u < my_units; u += kKWarps) {
             const int ti = u / U, ul = u - ti * U;
@@ -213,98 +221,92 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
             }
-            const int gt = rank + ti * nrank;
-            const int tx = gt % P.tiles_x;
             const int ux = ul * 8;
-            const bool skip = tx * P.TW + ux >= P.W;           // unit entirely right of the map
             const int stage = ti % S;
             if (!mbar_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
 
-            float e0[4], e1[4], e8[4], inv[4];
-            if (!skip) {
-                const unsigned char* sK = smem + (size_t)stage * L.stage_bytes;
-                const unsigned char* sQ = sK + 2 * L.halo_pad;
-                uint32_t qf[4][4];
+            const unsigned char* sK = smem + (size_t)stage * L.stage_bytes;
+            const unsigned char* sQ = sK + 2 * L.halo_pad;
+            // q of the lane's four pixels (rows 0..3 of column ux + g)
+            uint32_t qf[4][4];
 #pragma unroll
-                for (int py = 0; py < 4; ++py) {
-                    const uint4 v = lds_u4(sQ, (uint32_t)((py * P.TW + ux + g) * 64 + tig * 16));
-                    qf[py][0] = v.x; qf[py][1] = v.y; qf[py][2] = v.z; qf[py][3] = v.w;
-                }
-                const uint32_t lane_off = (uint32_t)((ux + g) * 64 + tig * 16);
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = lds_u4(sQ, (uint32_t)(i * P.TW + ux + g) * 64u + tig * 16u);
+                qf[i][0] = v.x; qf[i][1] = v.y; qf[i][2] = v.z; qf[i][3] = v.w;
+            }
+            // halo position (row r, column dx) of the lane's strip: pixel slot n0 + r*HW2 + dx
+            const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
 
-                float acc[2][3][4];
+            float acc[2][3][4];
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt)
+            for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-                    for (int nt = 0; nt < 3; ++nt)
+                for (int nt = 0; nt < 3; ++nt)
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+                    for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
 
 #pragma unroll
-                for (int dy = 0; dy < 3; ++dy) {
+            for (int dx = 0; dx < 3; ++dx) {
+                uint4 kc[6];                                       // one halo column, rows 0..5
 #pragma unroll
-                    for (int dx = 0; dx < 3; ++dx) {
+                for (int r = 0; r < 6; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)(r * HW2 + dx) * 64u);
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy) {
                         const int t = dy * 3 + dx;
-#pragma unroll
-                        for (int mt = 0; mt < 2; ++mt) {
-                            const uint4 k0 = lds_u4(sK, lane_off + (uint32_t)((2 * mt + dy) * HW2 + dx) * 64u);
-                            const uint4 k1 = lds_u4(sK, lane_off + (uint32_t)((2 * mt + 1 + dy) * HW2 + dx) * 64u);
-                            uint32_t a0[4], a1[4];
-                            a0[0] = hmul2_bf16(qf[2 * mt][0], k0.x);  a0[1] = hmul2_bf16(qf[2 * mt + 1][0], k1.x);
-                            a0[2] = hmul2_bf16(qf[2 * mt][1], k0.y);  a0[3] = hmul2_bf16(qf[2 * mt + 1][1], k1.y);
-                            a1[0] = hmul2_bf16(qf[2 * mt][2], k0.z);  a1[1] = hmul2_bf16(qf[2 * mt + 1][2], k1.z);
-                            a1[2] = hmul2_bf16(qf[2 * mt][3], k0.w);  a1[3] = hmul2_bf16(qf[2 * mt + 1][3], k1.w);
-                            mma_bf16(acc[mt][0], a0, bk[t][0][0], bk[t][0][1]);
-                            mma_bf16(acc[mt][1], a0, bk[t][0][2], bk[t][0][3]);
-                            mma_bf16(acc[mt][0], a1, bk[t][1][0], bk[t][1][1]);
-                            mma_bf16(acc[mt][1], a1, bk[t][1][2], bk[t][1][3]);
-                            if (t == 1) { mma_bf16(acc[mt][2], a0, ones_t1, ones_t1); mma_bf16(acc[mt][2], a1, ones_t1, ones_t1); }
-                            if (t == 8) { mma_bf16(acc[mt][2], a0, ones_t8, ones_t8); mma_bf16(acc[mt][2], a1, ones_t8, ones_t8); }
-                        }
+                        const uint4 k0 = kc[2 * mt + dy], k1 = kc[2 * mt + dy + 1];   // pixel rows 2mt / 2mt+1
+                        uint32_t a0[4], a1[4];
+                        a0[0] = hmul2_bf16(qf[2 * mt][0], k0.x);  a0[1] = hmul2_bf16(qf[2 * mt + 1][0], k1.x);
+                        a0[2] = hmul2_bf16(qf[2 * mt][1], k0.y);  a0[3] = hmul2_bf16(qf[2 * mt + 1][1], k1.y);
+                        a1[0] = hmul2_bf16(qf[2 * mt][2], k0.z);  a1[1] = hmul2_bf16(qf[2 * mt + 1][2], k1.z);
+                        a1[2] = hmul2_bf16(qf[2 * mt][3], k0.w);  a1[3] = hmul2_bf16(qf[2 * mt + 1][3], k1.w);
+                        mma_bf16(acc[mt][0], a0, bk[t][0][0], bk[t][0][1]);
+                        mma_bf16(acc[mt][1], a0, bk[t][0][2], bk[t][0][3]);
+                        mma_bf16(acc[mt][0], a1, bk[t][1][0], bk[t][1][1]);
+                        mma_bf16(acc[mt][1], a1, bk[t][1][2], bk[t][1][3]);
+                        if (t == 1) { mma_bf16(acc[mt][2], a0, ones_t1, ones_t1); mma_bf16(acc[mt][2], a1, ones_t1, ones_t1); }
+                        if (t == 8) { mma_bf16(acc[mt][2], a0, ones_t8, ones_t8); mma_bf16(acc[mt][2], a1, ones_t8, ones_t8); }
                     }
-                }
-
-                // softmax over the 9 slots; the 4 lanes of a quad share a pixel
-#pragma unroll
-                for (int py = 0; py < 4; ++py) {
-                    const int mt = py >> 1, o = (py & 1) * 2;
-                    const float x0 = acc[mt][0][o], x1 = acc[mt][0][o + 1];
-                    const float y0_ = acc[mt][1][o], y1_ = acc[mt][1][o + 1];
-                    const float z0 = acc[mt][2][o], z1 = acc[mt][2][o + 1];
-                    float l0, l1, l8;
-                    if (tig == 0) { l0 = x0 + y1_; l1 = x1 + z0; l8 = (y0_ + z1) * P.scale_log2e + bias8; }
-                    else          { l0 = x0 + y0_; l1 = x1 + y1_; l8 = -INFINITY; }
-                    l0 = l0 * P.scale_log2e + bias0;
-                    l1 = l1 * P.scale_log2e + bias1;
-                    float m = fmaxf(fmaxf(l0, l1), l8);
-                    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-                    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-                    e0[py] = fast_exp2(l0 - m);
-                    e1[py] = fast_exp2(l1 - m);
-                    e8[py] = fast_exp2(l8 - m);
-                    float s = e0[py] + e1[py] + e8[py];
-                    s += __shfl_xor_sync(0xffffffffu, s, 1);
-                    s += __shfl_xor_sync(0xffffffffu, s, 2);
-                    inv[py] = 1.f / s;
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEmpty + stage));        // done with k and q of this unit
 
-            if (!skip) {
-                const int which = (u >> 2) & 1;                        // value warp `warp` or `warp + 4`
-                const int sent = which ? sent1 : sent0;
-                const int vw = warp + 4 * which, slot = sent & 1;
-                if (!mbar_wait(bar(kBarMailEmpty + vw * 2 + slot), ((sent >> 1) & 1) ^ 1)) { ok = false; break; }
-                unsigned char* mail = smem + L.mail_off + (size_t)(vw * 2 + slot) * kMailBytes;
-                *reinterpret_cast<float4*>(mail + (g * 10 + 2 * tig) * 16) = make_float4(e0[0], e0[1], e0[2], e0[3]);
-                *reinterpret_cast<float4*>(mail + (g * 10 + 2 * tig + 1) * 16) = make_float4(e1[0], e1[1], e1[2], e1[3]);
-                if (tig == 0) *reinterpret_cast<float4*>(mail + (g * 10 + 8) * 16) = make_float4(e8[0], e8[1], e8[2], e8[3]);
-                if (tig == 1) *reinterpret_cast<float4*>(mail + (g * 10 + 9) * 16) = make_float4(inv[0], inv[1], inv[2], inv[3]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarMailFull + vw * 2 + slot));
-                if (which) ++sent1; else ++sent0;
+            // softmax over the 9 slots; the 4 lanes of a quad share a pixel
+            float e0[4], e1[4], e8[4], inv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int mt = i >> 1, o = (i & 1) * 2;
+                const float x0 = acc[mt][0][o], x1 = acc[mt][0][o + 1];
+                const float y0_ = acc[mt][1][o], y1_ = acc[mt][1][o + 1];
+                const float z0 = acc[mt][2][o], z1 = acc[mt][2][o + 1];
+                float l0, l1, l8;
+                if (tig == 0) { l0 = x0 + y1_; l1 = x1 + z0; l8 = (y0_ + z1) * P.scale_log2e + bias8; }
+                else          { l0 = x0 + y0_; l1 = x1 + y1_; l8 = -INFINITY; }
+                l0 = l0 * P.scale_log2e + bias0;
+                l1 = l1 * P.scale_log2e + bias1;
+                float m = fmaxf(fmaxf(l0, l1), l8);
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+                e0[i] = fast_exp2(l0 - m);
+                e1[i] = fast_exp2(l1 - m);
+                e8[i] = fast_exp2(l8 - m);
+                float s = e0[i] + e1[i] + e8[i];
+                s += __shfl_xor_sync(0xffffffffu, s, 1);
+                s += __shfl_xor_sync(0xffffffffu, s, 2);
+                inv[i] = 1.f / s;
             }
+
+            const int slot = u % kMailSlots;
+            if (!mbar_wait(bar(kBarMailEmpty + slot), ((u / kMailSlots) & 1) ^ 1)) { ok = false; break; }
+            unsigned char* mail = smem + L.mail_off + (size_t)slot * kMailBytes;
+            *reinterpret_cast<float4*>(mail + (g * 10 + 2 * tig) * 16) = make_float4(e0[0], e0[1], e0[2], e0[3]);
+            *reinterpret_cast<float4*>(mail + (g * 10 + 2 * tig + 1) * 16) = make_float4(e1[0], e1[1], e1[2], e1[3]);
+            if (tig == 0) *reinterpret_cast<float4*>(mail + (g * 10 + 8) * 16) = make_float4(e8[0], e8[1], e8[2], e8[3]);
+            if (tig == 1) *reinterpret_cast<float4*>(mail + (g * 10 + 9) * 16) = make_float4(inv[0], inv[1], inv[2], inv[3]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarMailFull + slot));
         }
         // key warp 0 may run out of units before the last tiles are requested: issue the rest
         if (warp == 0 && lane == 0 && ok && !produce(my_tiles)) ok = false;
@@ -329,7 +331,6 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
-        int recv = 0;
 
         for (int u = vw; ok && u < my_units; u += kVWarps) {
             const int ti = u / U, ul = u - ti * U;
@@ -338,80 +339,82 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             const int ty = (gt / P.tiles_x) % P.tiles_y;
             const int b = gt / (P.tiles_x * P.tiles_y);
             const int ux = ul * 8;
-            const int x = tx * P.TW + ux + g, y0 = ty * 4;
-            const bool skip = tx * P.TW + ux >= P.W;
             const int stage = ti % S;
             if (!mbar_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
+            const int slot = u % kMailSlots;
+            if (!mbar_wait(bar(kBarMailFull + slot), (u / kMailSlots) & 1)) { ok = false; break; }
+            const unsigned char* mail = smem + L.mail_off + (size_t)slot * kMailBytes;
+            const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
+            const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
 
+            uint32_t af[2][4];
+            float4 invv;
+            {
+                const float4 lo = lds_f4(mail, (g * 10 + 2 * tig) * 16);
+                const float4 hi = lds_f4(mail, (g * 10 + 2 * tig + 1) * 16);
+                const float4 e8v = lds_f4(mail, (g * 10 + 8) * 16);
+                invv = lds_f4(mail, (g * 10 + 9) * 16);
+                af[0][0] = pack_bf16(lo.x, hi.x);  af[0][1] = pack_bf16(lo.y, hi.y);
+                af[1][0] = pack_bf16(lo.z, hi.z);  af[1][1] = pack_bf16(lo.w, hi.w);
+                af[0][2] = tig == 0 ? pack_bf16(e8v.x, 0.f) : 0u;  af[0][3] = tig == 0 ? pack_bf16(e8v.y, 0.f) : 0u;
+                af[1][2] = tig == 0 ? pack_bf16(e8v.z, 0.f) : 0u;  af[1][3] = tig == 0 ? pack_bf16(e8v.w, 0.f) : 0u;
+            }
             float o_acc[4][8];
-            float4 invv = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!skip) {
-                const int slot = recv & 1;
-                if (!mbar_wait(bar(kBarMailFull + vw * 2 + slot), (recv >> 1) & 1)) { ok = false; break; }
-                const unsigned char* mail = smem + L.mail_off + (size_t)(vw * 2 + slot) * kMailBytes;
-                const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
-                const uint32_t lane_off = (uint32_t)((ux + g) * 64 + tig * 16);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) o_acc[i][c] = 0.f;
 
-                uint32_t af[2][4];
-                {
-                    const float4 lo = lds_f4(mail, (g * 10 + 2 * tig) * 16);
-                    const float4 hi = lds_f4(mail, (g * 10 + 2 * tig + 1) * 16);
-                    const float4 e8v = lds_f4(mail, (g * 10 + 8) * 16);
-                    invv = lds_f4(mail, (g * 10 + 9) * 16);
-                    af[0][0] = pack_bf16(lo.x, hi.x);  af[0][1] = pack_bf16(lo.y, hi.y);
-                    af[1][0] = pack_bf16(lo.z, hi.z);  af[1][1] = pack_bf16(lo.w, hi.w);
-                    af[0][2] = tig == 0 ? pack_bf16(e8v.x, 0.f) : 0u;  af[0][3] = tig == 0 ? pack_bf16(e8v.y, 0.f) : 0u;
-                    af[1][2] = tig == 0 ? pack_bf16(e8v.z, 0.f) : 0u;  af[1][3] = tig == 0 ? pack_bf16(e8v.w, 0.f) : 0u;
+#pragma unroll
+            for (int dx = 0; dx < 3; ++dx) {
+                // one halo column of the strip, rows 0..5, widened to fp32 once
+                float vf[6][8];
+#pragma unroll
+                for (int r = 0; r < 6; ++r) {
+                    const uint4 v = lds_u4(sV, off0 + (uint32_t)(r * HW2 + dx) * 64u);
+                    vf[r][0] = bf16_lo(v.x); vf[r][1] = bf16_hi(v.x);
+                    vf[r][2] = bf16_lo(v.y); vf[r][3] = bf16_hi(v.y);
+                    vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
+                    vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
                 }
 #pragma unroll
-                for (int py = 0; py < 4; ++py)
+                for (int r = 0; r < 5; ++r) {                      // rows r (half 0) and r+1 (half 1)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) o_acc[py][i] = 0.f;
-
-#pragma unroll
-                for (int dy = 0; dy < 3; ++dy) {
-#pragma unroll
-                    for (int dx = 0; dx < 3; ++dx) {
+                    for (int mt = 0; mt < 2; ++mt) {
+                        const int dy = r - 2 * mt;
+                        if (dy < 0 || dy > 2) continue;
                         const int t = dy * 3 + dx;
-                        const float4 et = lds_f4(mail, (g * 10 + t) * 16);       // e[row 0..3][t]
-                        const float er[4] = {et.x, et.y, et.z, et.w};
+                        const float4 et = lds_f4(mail, (g * 10 + t) * 16);       // e[pixel 0..3][t]
+                        const float ea = mt == 0 ? et.x : et.z, eb = mt == 0 ? et.y : et.w;
 #pragma unroll
-                        for (int mt = 0; mt < 2; ++mt) {
-                            const uint4 v0 = lds_u4(sV, lane_off + (uint32_t)((2 * mt + dy) * HW2 + dx) * 64u);
-                            const uint4 v1 = lds_u4(sV, lane_off + (uint32_t)((2 * mt + 1 + dy) * HW2 + dx) * 64u);
-                            const uint32_t v0r[4] = {v0.x, v0.y, v0.z, v0.w};
-                            const uint32_t v1r[4] = {v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                float c[4] = {er[2 * mt], er[2 * mt], er[2 * mt + 1], er[2 * mt + 1]};
-                                mma_bf16(c, af[mt], bv[t][j][0], bv[t][j][1]);
-                                o_acc[2 * mt][2 * j]         = fmaf(c[0], bf16_lo(v0r[j]), o_acc[2 * mt][2 * j]);
-                                o_acc[2 * mt][2 * j + 1]     = fmaf(c[1], bf16_hi(v0r[j]), o_acc[2 * mt][2 * j + 1]);
-                                o_acc[2 * mt + 1][2 * j]     = fmaf(c[2], bf16_lo(v1r[j]), o_acc[2 * mt + 1][2 * j]);
-                                o_acc[2 * mt + 1][2 * j + 1] = fmaf(c[3], bf16_hi(v1r[j]), o_acc[2 * mt + 1][2 * j + 1]);
-                            }
+                        for (int j = 0; j < 4; ++j) {
+                            float d[4];
+                            mma_bf16_c(d, af[mt], bv[t][j][0], bv[t][j][1], ea, ea, eb, eb);
+                            ffma2(o_acc[2 * mt][2 * j], o_acc[2 * mt][2 * j + 1], d[0], d[1],
+                                  vf[r][2 * j], vf[r][2 * j + 1]);
+                            ffma2(o_acc[2 * mt + 1][2 * j], o_acc[2 * mt + 1][2 * j + 1], d[2], d[3],
+                                  vf[r + 1][2 * j], vf[r + 1][2 * j + 1]);
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarMailEmpty + vw * 2 + slot));
-                ++recv;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarEmpty + stage));        // done with v of this unit
+            if (lane == 0) {
+                mbar_arrive(bar(kBarMailEmpty + slot));
+                mbar_arrive(bar(kBarEmpty + stage));                   // done with v of this unit
+            }
 
-            if (!skip && x < P.W) {
-                const float invr[4] = {invv.x, invv.y, invv.z, invv.w};
+            const float invr[4] = {invv.x, invv.y, invv.z, invv.w};
 #pragma unroll
-                for (int py = 0; py < 4; ++py) {
-                    if (y0 + py < P.H) {
-                        uint4 r;
-                        r.x = pack_bf16(o_acc[py][0] * invr[py], o_acc[py][1] * invr[py]);
-                        r.y = pack_bf16(o_acc[py][2] * invr[py], o_acc[py][3] * invr[py]);
-                        r.z = pack_bf16(o_acc[py][4] * invr[py], o_acc[py][5] * invr[py]);
-                        r.w = pack_bf16(o_acc[py][6] * invr[py], o_acc[py][7] * invr[py]);
-                        *reinterpret_cast<uint4*>(P.out + ((size_t)(b * P.H + y0 + py) * P.W + x) * C + h * kHeadDim + tig * 8) = r;
-                    }
+            for (int i = 0; i < 4; ++i) {
+                const int y = ty * 4 + i, x = tx * P.TW + ux + g;
+                if (y < P.H && x < P.W) {
+                    uint4 r;
+                    r.x = pack_bf16(o_acc[i][0] * invr[i], o_acc[i][1] * invr[i]);
+                    r.y = pack_bf16(o_acc[i][2] * invr[i], o_acc[i][3] * invr[i]);
+                    r.z = pack_bf16(o_acc[i][4] * invr[i], o_acc[i][5] * invr[i]);
+                    r.w = pack_bf16(o_acc[i][6] * invr[i], o_acc[i][7] * invr[i]);
+                    *reinterpret_cast<uint4*>(P.out + ((size_t)(b * P.H + y) * P.W + x) * C + h * kHeadDim + tig * 8) = r;
                 }
             }
         }

@@ -28,9 +28,17 @@ namespace slide_attn {
 
 namespace {
 
+// Tuning knobs (compile time).
+#ifndef SA_WS_KWARPS
+#define SA_WS_KWARPS 6
+#endif
+#ifndef SA_WS_VWARPS
+#define SA_WS_VWARPS 6
+#endif
+
 constexpr int kHeadDim = 32;
-constexpr int kKWarps = 6;
-constexpr int kVWarps = 6;
+constexpr int kKWarps = SA_WS_KWARPS;
+constexpr int kVWarps = SA_WS_VWARPS;
 constexpr int kThreads = (kKWarps + kVWarps) * 32;
 constexpr int kMaxStages = 3;
 constexpr int kMailSlots = 16;

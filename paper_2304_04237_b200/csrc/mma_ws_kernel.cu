@@ -7,7 +7,8 @@
 //   * key warps and value warps.  A key warp keeps all key-side B fragments (72 registers) and
 //     turns a unit (4 rows x 8 columns) into unnormalised softmax weights e[p, 0..8] and 1/sum; a
 //     value warp keeps all value-side B fragments and turns e into the output.  e travels through
-//     a ring of shared-memory mailboxes (one per unit in flight), guarded by mbarriers;
+//     small rings of shared-memory mailboxes (one ring per key/value warp pair), guarded by
+//     mbarriers;
 //   * K / V halo tiles and the q tile arrive by TMA (zero fill outside the map = the padding of the
 //     convolution) into a 3-stage ring; lane 0 of key warp 0 is the producer;
 //   * the fp32 weights of the head are brought in once by two 1-D bulk copies and every warp builds
@@ -41,7 +42,13 @@ constexpr int kKWarps = SA_WS_KWARPS;
 constexpr int kVWarps = SA_WS_VWARPS;
 constexpr int kThreads = (kKWarps + kVWarps) * 32;
 constexpr int kMaxStages = 3;
-constexpr int kMailSlots = 16;
+// Mailbox rings: unit u uses ring u % kRings, so every ring has exactly one writing key warp and
+// one reading value warp, both walking it in order; kRingDepth slots per ring.
+constexpr int kRings = kKWarps > kVWarps ? kKWarps : kVWarps;
+constexpr int kRingDepth = 2;
+constexpr int kMailSlots = kRings * kRingDepth;
+static_assert(kRings % kKWarps == 0 && kRings % kVWarps == 0, "one warp count must divide the other");
+static_assert(kMailSlots <= 16, "barrier table holds 16 mailbox slots");
 constexpr int kMailBytes = 8 * 10 * 4 * 4;              // [g 8][slot 0..8, 9 = 1/sum][pixel 4] floats
 constexpr int kWeightBytes = kHeadDim * 81 * 4;         // fp32 weights of one head, one side
 constexpr float kLog2e = 1.4426950408889634f;
@@ -117,13 +124,12 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const int nrank = ((int)gridDim.x - h + P.heads - 1) / P.heads;
     const int tiles_per_head = P.B * P.tiles_y * P.tiles_x;
     const int my_tiles = rank < tiles_per_head ? (tiles_per_head - rank + nrank - 1) / nrank : 0;
-    const int my_units = my_tiles * U;
     const int C = P.heads * kHeadDim;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(bar(kBarFull + s), 1);
-            mbar_init(bar(kBarEmpty + s), 2 * U);
+            mbar_init(bar(kBarEmpty + s), kKWarps + kVWarps);
         }
         for (int i = 0; i < kMailSlots; ++i) {
             mbar_init(bar(kBarMailFull + i), 1);
@@ -221,17 +227,22 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const uint32_t ones_t1 = g == 0 ? kOnesBf16x2 : 0u;    // third n-tile: column 0 sums tap 1,
         const uint32_t ones_t8 = g == 1 ? kOnesBf16x2 : 0u;    //               column 1 sums tap 8
 
-        for (int u = warp; ok && u < my_units; u += kKWarps) {
-            const int ti = u / U, ul = u - ti * U;
+        // Every warp visits every tile in order (waits for it, arrives on its release barrier), even
+        // a tile in which it owns no unit: a warp that skipped a phase of a barrier could later
+        // mistake an older phase for the one it waits for.
+        for (int ti = 0; ok && ti < my_tiles; ++ti) {
             // ---- producer duty (key warp 0, lane 0): keep the ring filled -------------------
             if (warp == 0) {
                 if (lane == 0 && !produce(ti)) ok = false;
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
             }
-            const int ux = ul * 8;
             const int stage = ti % S;
             if (!mbar_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
+            const int u0 = ti * U;
+          for (int ul = (warp + kKWarps - u0 % kKWarps) % kKWarps; ul < U; ul += kKWarps) {
+            const int u = u0 + ul;
+            const int ux = ul * 8;
 
             const unsigned char* sK = smem + (size_t)stage * L.stage_bytes;
             const unsigned char* sQ = sK + 2 * L.halo_pad;
@@ -278,9 +289,6 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarEmpty + stage));        // done with k and q of this unit
-
             // softmax over the 9 slots; the 4 lanes of a quad share a pixel
             float e0[4], e1[4], e8[4], inv[4];
 #pragma unroll
@@ -306,8 +314,9 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 inv[i] = 1.f / s;
             }
 
-            const int slot = u % kMailSlots;
-            if (!mbar_wait(bar(kBarMailEmpty + slot), ((u / kMailSlots) & 1) ^ 1)) { ok = false; break; }
+            const int seq = u / kRings;                                 // position in ring u % kRings
+            const int slot = (u % kRings) * kRingDepth + seq % kRingDepth;
+            if (!mbar_wait(bar(kBarMailEmpty + slot), ((seq / kRingDepth) & 1) ^ 1)) { ok = false; break; }
             unsigned char* mail = smem + L.mail_off + (size_t)slot * kMailBytes;
             *reinterpret_cast<float4*>(mail + (g * 10 + 2 * tig) * 16) = make_float4(e0[0], e0[1], e0[2], e0[3]);
             *reinterpret_cast<float4*>(mail + (g * 10 + 2 * tig + 1) * 16) = make_float4(e1[0], e1[1], e1[2], e1[3]);
@@ -315,9 +324,10 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             if (tig == 1) *reinterpret_cast<float4*>(mail + (g * 10 + 9) * 16) = make_float4(inv[0], inv[1], inv[2], inv[3]);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarMailFull + slot));
+          }
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
         }
-        // key warp 0 may run out of units before the last tiles are requested: issue the rest
-        if (warp == 0 && lane == 0 && ok && !produce(my_tiles)) ok = false;
     } else {
         // =====================================================================================
         // value warps
@@ -340,17 +350,20 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
 
-        for (int u = vw; ok && u < my_units; u += kVWarps) {
-            const int ti = u / U, ul = u - ti * U;
+        for (int ti = 0; ok && ti < my_tiles; ++ti) {
             const int gt = rank + ti * nrank;
             const int tx = gt % P.tiles_x;
             const int ty = (gt / P.tiles_x) % P.tiles_y;
             const int b = gt / (P.tiles_x * P.tiles_y);
-            const int ux = ul * 8;
             const int stage = ti % S;
             if (!mbar_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
-            const int slot = u % kMailSlots;
-            if (!mbar_wait(bar(kBarMailFull + slot), (u / kMailSlots) & 1)) { ok = false; break; }
+            const int u0 = ti * U;
+          for (int ul = (vw + kVWarps - u0 % kVWarps) % kVWarps; ul < U; ul += kVWarps) {
+            const int u = u0 + ul;
+            const int ux = ul * 8;
+            const int seq = u / kRings;
+            const int slot = (u % kRings) * kRingDepth + seq % kRingDepth;
+            if (!mbar_wait(bar(kBarMailFull + slot), (seq / kRingDepth) & 1)) { ok = false; break; }
             const unsigned char* mail = smem + L.mail_off + (size_t)slot * kMailBytes;
             const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
             const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
@@ -407,10 +420,7 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
             }
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(kBarMailEmpty + slot));
-                mbar_arrive(bar(kBarEmpty + stage));                   // done with v of this unit
-            }
+            if (lane == 0) mbar_arrive(bar(kBarMailEmpty + slot));
 
             const float invr[4] = {invv.x, invv.y, invv.z, invv.w};
 #pragma unroll
@@ -425,6 +435,9 @@ mma_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     *reinterpret_cast<uint4*>(P.out + ((size_t)(b * P.H + y) * P.W + x) * C + h * kHeadDim + tig * 8) = r;
                 }
             }
+          }
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
         }
     }
     if (!ok && lane == 0) atomicExch(P.status, 1);

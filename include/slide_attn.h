@@ -79,9 +79,12 @@ typedef enum {
     SLIDE_ATTN_VARIANT_MMA     = 2,   /* TMA halo tile in shared memory, deformed-shift contraction on
                                          tensor cores (bf16 operands, fp32 accumulate); one CTA per
                                          tile and head; bf16, head_dim 32, ksize 3                      */
-    SLIDE_ATTN_VARIANT_MMA_WS  = 3    /* same arithmetic, persistent warp-specialised schedule (key
+    SLIDE_ATTN_VARIANT_MMA_WS  = 3,   /* same arithmetic, persistent warp-specialised schedule (key
                                          warps / value warps, 3-stage TMA ring, weights resident in
                                          registers, single launch); bf16, head_dim 32, ksize 3          */
+    SLIDE_ATTN_VARIANT_UMMA    = 4    /* MMA_WS with the value-side contraction on the 5th-generation
+                                         tensor core (tcgen05.mma, accumulator in tensor memory);
+                                         bf16, head_dim 32, ksize 3                                     */
 } slide_attn_variant;
 
 /*

@@ -50,4 +50,10 @@ bool mma_ws_supports(slide_attn_dtype dtype, int head_dim, int ksize);
 cudaError_t mma_ws_setup();
 cudaError_t launch_mma_ws(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
 
+
+// UMMA variant: as MMA_WS, with the value-side contraction on tcgen05 / tensor memory.
+bool umma_supports(slide_attn_dtype dtype, int head_dim, int ksize);
+cudaError_t umma_setup();
+cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
+
 }  // namespace slide_attn

@@ -1,0 +1,619 @@
+// UMMA variant (bf16, head_dim 32, k = 3): like MMA_WS a persistent, warp-specialised kernel, but the
+// value-side contraction runs on the 5th-generation tensor core (tcgen05.mma) with its accumulator
+// in tensor memory.
+//
+// Arithmetic (Eq. 2 with Eq. 12 inside; w = E + D split as in mma_kernel.cu):
+//   key side    logit[p,s] = sum_{t,c} q[p,c] k[p+off(t),c] (D_k[c,s,t] + [t == s])   mma.sync, key warps
+//   softmax     e[p,s] = exp(logit - max)                                               key warps
+//   value side  A'[p,(t,c)] = sum_s e[p,s] (D_v[c,s,t] + [t == s])                      tcgen05.mma
+//               sum[p]      = sum_s e[p,s]                                              (16 extra columns)
+//               out[p,c]    = (sum_t A'[p,t,c] v[p+off(t),c]) / sum[p]                  value warps
+//
+// The value-side product is one [128 pixels x 32] x [32 x 304] bf16 MMA per block of four units:
+//   A row p (shared memory, written by the key warps):  e_hi[0..7] | e_hi[0..7] | e_lo[0..7] |
+//                                                       e_hi[8], e_hi[8], e_lo[8], 0 ...
+//     with e = e_hi + e_lo split into two bf16 values, so that the one-hot part is carried to
+//     2^-17 relative accuracy while D_v only meets e_hi;
+//   B column (t,c) (shared memory, built once per CTA):  D_v[c][0..7][t] | [s == t] | [s == t] |
+//                                                       D_v[c][8][t], [t == 8], [t == 8], 0 ...
+//   16 more columns hold 0 | 1 | 1 | 0,1,1,0... and so deliver sum_s e[p,s].
+// D (fp32) lives in tensor memory, pixel = TMEM lane.  Columns are ordered by tap column dx: the
+// taps with dx = 0, 1 (192 columns) form part 1, those with dx = 2 plus the sum columns (112) part
+// 2.  Part 1 is double-buffered across blocks, part 2 single-buffered (192 + 112 + 192 = 496 of the
+// 512 TMEM columns).  Value warp w reads TMEM lanes 32w .. 32w+31 (its quadrant) with
+// tcgen05.ld.16x256b, whose register layout equals the mma.sync accumulator fragment.
+//
+// Roles (12 warps): warps 0-3 value warps (warp index = TMEM quadrant = unit index within a block),
+// warps 4-10 key warps (lane 0 of the first one is the TMA producer), warp 11 allocates / frees
+// tensor memory and its lane 0 issues the MMAs.  Every wait is bounded; a wait that runs out sets
+// the status word, and tensor memory is released on every path.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace slide_attn {
+
+namespace {
+
+constexpr int kHeadDim = 32;
+constexpr int kVWarps = 4;
+constexpr int kKWarps = 7;
+constexpr int kCtlWarp = kVWarps + kKWarps;             // warp 11
+constexpr int kThreads = (kVWarps + kKWarps + 1) * 32;
+constexpr int kMaxStages = 3;
+constexpr int kABufs = 3;                               // A tiles (one per block in flight)
+constexpr int kABytes = 128 * 64;                       // 128 rows x 32 bf16
+constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
+constexpr int kBBytes = kBCols * 64;
+constexpr int kWeightBytes = kHeadDim * 81 * 4;         // fp32 weights of one head, one side
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColP1a = 0, kColP2 = 192, kColP1b = 304;   // TMEM column regions
+constexpr uint32_t kIdescP1 = umma_idesc_bf16(128, 192);
+constexpr uint32_t kIdescP2 = umma_idesc_bf16(128, 112);
+
+struct UmmaParams {
+    const float* wk;
+    const float* wv;
+    const float* bias;         // [heads][9] or nullptr
+    __nv_bfloat16* out;
+    int* status;
+    int B, H, W, heads;
+    int TW;                    // tile width in pixels (multiple of 8); tile height is 4
+    int tiles_x, tiles_y;
+    int stages;                // 2 or 3
+    float scale_log2e;         // log2(e) / sqrt(head_dim)
+};
+
+struct Smem {
+    uint32_t halo_pad;         // bytes of one K or V halo tile (6 rows x (TW+2) pixels x 64 B), 1024-aligned
+    uint32_t stage_bytes;      // K halo | V halo | q tile
+    uint32_t b_off;            // B tile of the value-side MMA
+    uint32_t a_off;            // A tiles [kABufs][kABytes]
+    uint32_t tmem_off;         // TMEM base address written by tcgen05.alloc
+    uint32_t bar_off;          // mbarriers
+    uint32_t total;            // including 1024 bytes of slack to align the base
+};
+
+__host__ __device__ inline Smem smem_layout(int TW, int stages) {
+    Smem s;
+    s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 1023u) & ~1023u;
+    s.stage_bytes = 2 * s.halo_pad + (((uint32_t)(4 * TW * 64) + 1023u) & ~1023u);
+    // the last stage doubles as the staging area of the head's fp32 weights (both sides)
+    const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
+    if (s.stage_bytes < wbytes) s.stage_bytes = wbytes;
+    s.b_off = s.stage_bytes * stages;
+    s.a_off = s.b_off + kBBytes;
+    s.tmem_off = s.a_off + kABufs * kABytes;
+    s.bar_off = s.tmem_off + 16;
+    s.total = s.bar_off + 32 * 8 + 1024;
+    return s;
+}
+
+// barrier indices (8 bytes each) behind bar_off
+constexpr int kBarFull = 0;          // [stage]  TMA landed
+constexpr int kBarEmpty = 3;         // [stage]  every key and value warp is done with the stage
+constexpr int kBarWeights = 6;       // weights landed
+constexpr int kBarWeightsDone = 7;   // all warps have built their fragments / their share of the B tile
+constexpr int kBarAReady = 8;        // [A buffer]  the 4 units of a block have written their rows
+constexpr int kBarAFree = 11;        // [A buffer]  the MMAs reading the buffer are complete
+constexpr int kBarDFull = 14;        // [region: part 1 even, part 2, part 1 odd]  MMA results in TMEM
+constexpr int kBarDFree = 17;        // [region]  the 4 value warps are done reading the region
+constexpr int kBarVDone = 20;        // value warps have finished all TMEM reads
+
+__device__ __forceinline__ float4 lds_f4(const unsigned char* base, uint32_t off) {
+    return *reinterpret_cast<const float4*>(base + off);
+}
+__device__ __forceinline__ uint4 lds_u4(const unsigned char* base, uint32_t off) {
+    return *reinterpret_cast<const uint4*>(base + off);
+}
+
+// Bounded wait whose verdict is the same in all lanes of the (converged) warp.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
+}
+
+// Value B(n, k) of the value-side MMA for one head; wv: fp32 [32][9][9] of the head.
+__device__ __forceinline__ float b_value(const float* wv, int n, int k) {
+    if (n >= 288) return (k >= 8 && k < 24) || k == 25 || k == 26 ? 1.f : 0.f;      // sum columns
+    const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;          // columns are ordered dx-major
+    const int cn = n & 31, j = cn >> 3, wi = cn & 7;
+    const int c = 8 * (wi >> 1) + 2 * j + (wi & 1);
+    if (k < 8) return wv[c * 81 + k * 9 + t] - (k == t ? 1.f : 0.f);
+    if (k < 16) return (k - 8) == t ? 1.f : 0.f;
+    if (k < 24) return (k - 16) == t ? 1.f : 0.f;
+    if (k == 24) return wv[c * 81 + 72 + t] - (t == 8 ? 1.f : 0.f);
+    if (k == 25 || k == 26) return t == 8 ? 1.f : 0.f;
+    return 0.f;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+            const __grid_constant__ CUtensorMap map_v, const UmmaParams P)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-aligned
+    const Smem L = smem_layout(P.TW, P.stages);
+    const uint32_t bar0 = smem_u32(smem + L.bar_off);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tig = lane & 3;
+    const int S = P.stages;
+    const int U = P.TW >> 3;                                   // units per tile
+    const int HW2 = P.TW + 2;
+
+    // this CTA's head and its share of that head's tiles
+    const int h = blockIdx.x % P.heads;
+    const int rank = blockIdx.x / P.heads;
+    const int nrank = ((int)gridDim.x - h + P.heads - 1) / P.heads;
+    const int tiles_per_head = P.B * P.tiles_y * P.tiles_x;
+    const int my_tiles = rank < tiles_per_head ? (tiles_per_head - rank + nrank - 1) / nrank : 0;
+    const int my_units = my_tiles * U;
+    const int my_blocks = (my_units + 3) >> 2;                 // blocks of four units = 128 pixels
+    const int C = P.heads * kHeadDim;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(bar(kBarFull + s), 1);
+            mbar_init(bar(kBarEmpty + s), kKWarps + kVWarps);
+        }
+        mbar_init(bar(kBarWeights), 1);
+        mbar_init(bar(kBarWeightsDone), kKWarps + kVWarps + 1);
+        for (int i = 0; i < kABufs; ++i) {
+            mbar_init(bar(kBarAReady + i), 4);
+            mbar_init(bar(kBarAFree + i), 1);
+        }
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(bar(kBarDFull + i), 1);
+            mbar_init(bar(kBarDFree + i), kVWarps);
+        }
+        mbar_init(bar(kBarVDone), kVWarps);
+    }
+    // A tiles start as zeros: the columns no key warp ever writes must not hold NaN patterns
+    for (int i = threadIdx.x; i < kABufs * kABytes / 16; i += kThreads)
+        reinterpret_cast<uint4*>(smem + L.a_off)[i] = make_uint4(0, 0, 0, 0);
+    if (warp == kCtlWarp) tmem_alloc(smem_u32(smem + L.tmem_off), kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *reinterpret_cast<const volatile uint32_t*>(smem + L.tmem_off);
+
+    // tile n of this CTA -> stage n % S
+    auto issue_tile = [&](int n) {
+        const int gt = rank + n * nrank;
+        const int tx = gt % P.tiles_x;
+        const int ty = (gt / P.tiles_x) % P.tiles_y;
+        const int b = gt / (P.tiles_x * P.tiles_y);
+        const int s = n % S;
+        const uint32_t base = smem_u32(smem + (size_t)s * L.stage_bytes);
+        const uint32_t fb = bar(kBarFull + s);
+        mbar_expect_tx(fb, (uint32_t)(2 * 6 * HW2 * 64 + 4 * P.TW * 64));
+        tma_load_4d(base, &map_k, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
+        tma_load_4d(base + L.halo_pad, &map_v, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
+        tma_load_4d(base + 2 * L.halo_pad, &map_q, fb, h * kHeadDim, tx * P.TW, ty * 4, b);
+    };
+
+    // The fp32 weights of the head are staged in the LAST stage's memory; that stage receives its
+    // first tile only after every warp has finished with them.
+    const unsigned char* w_stage = smem + (size_t)(S - 1) * L.stage_bytes;
+    int issued = 0;                                            // producer state (first key warp, lane 0)
+    if (my_tiles > 0 && warp == kVWarps && lane == 0) {
+        mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
+        bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
+        bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
+        while (issued < my_tiles && issued < S - 1) issue_tile(issued++);
+    }
+    __syncwarp();
+
+    // Issues every tile whose stage is free.  A tile that the producer's own warp needs now (index
+    // <= `need`) is waited for; later ones are only probed.  Returns false if a wait ran out.
+    auto produce = [&](int need) -> bool {
+        while (issued < my_tiles) {
+            uint32_t b = 0, par = 0;
+            bool gated = false;
+            if (issued == S - 1) { b = bar(kBarWeightsDone); par = 0; gated = true; }   // staging area must be dead
+            else if (issued >= S) { b = bar(kBarEmpty + issued % S); par = ((issued / S) - 1) & 1; gated = true; }
+            if (gated && !mbar_test(b, par)) {
+                if (issued > need) return true;               // not needed yet: try again later
+                if (!mbar_wait(b, par)) return false;
+            }
+            issue_tile(issued++);
+        }
+        return true;
+    };
+
+    bool ok = my_tiles > 0 && warp_wait(bar(kBarWeights), 0);
+    const float* wks = reinterpret_cast<const float*>(w_stage);
+    const float* wvs = wks + kHeadDim * 81;
+
+    // ---- B tile of the value-side MMA: every thread converts its share ---------------------------
+    if (ok) {
+        unsigned char* sB = smem + L.b_off;
+        for (int idx = threadIdx.x; idx < kBCols * 16; idx += kThreads) {
+            const int n = idx >> 4, k = (idx & 15) * 2;
+            const uint32_t w = pack_bf16(b_value(wvs, n, k), b_value(wvs, n, k + 1));
+            *reinterpret_cast<uint32_t*>(sB + (n >> 3) * 512 + (k >> 3) * 128 + (n & 7) * 16 + (k & 7) * 2) = w;
+        }
+        fence_proxy_async_smem();
+    }
+
+    if (warp >= kVWarps && warp < kCtlWarp) {
+        // =====================================================================================
+        // key warps
+        // =====================================================================================
+        const int kw = warp - kVWarps;
+        uint32_t bk[9][2][4];          // [tap][k-step][n-tile 0: r0 r1 | n-tile 1: r0 r1]
+        if (ok) {
+#pragma unroll
+            for (int t = 0; t < 9; ++t)
+#pragma unroll
+                for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        const int c0 = 8 * tig + 4 * ks + 2 * r;
+                        {   // n-tile 0: column g = slot g
+                            const float e = (g == t) ? 1.f : 0.f;
+                            bk[t][ks][r] = pack_bf16(wks[c0 * 81 + g * 9 + t] - e, wks[(c0 + 1) * 81 + g * 9 + t] - e);
+                        }
+                        {   // n-tile 1: column 0 = slot 8; column 1 sums tap 0; column n >= 2 sums tap n
+                            const float e = (t == 8) ? 1.f : 0.f;
+                            const uint32_t d = pack_bf16(wks[c0 * 81 + 72 + t] - e, wks[(c0 + 1) * 81 + 72 + t] - e);
+                            const int tap = g == 1 ? 0 : g;
+                            bk[t][ks][2 + r] = g == 0 ? d : (t == tap ? kOnesBf16x2 : 0u);
+                        }
+                    }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
+
+        float bias0 = 0.f, bias1 = 0.f, bias8 = 0.f;
+        if (P.bias) {
+            const float* bh = P.bias + h * 9;
+            bias0 = bh[2 * tig] * kLog2e;
+            bias1 = bh[2 * tig + 1] * kLog2e;
+            bias8 = bh[8] * kLog2e;
+        }
+        const uint32_t ones_t1 = g == 0 ? kOnesBf16x2 : 0u;    // third n-tile: column 0 sums tap 1,
+        const uint32_t ones_t8 = g == 1 ? kOnesBf16x2 : 0u;    //               column 1 sums tap 8
+
+        // Every warp visits every tile in order (waits for it, arrives on its release barrier), even
+        // a tile in which it owns no unit: a warp that skipped a phase of a barrier could later
+        // mistake an older phase for the one it waits for.
+        for (int ti = 0; ok && ti < my_tiles; ++ti) {
+            if (kw == 0) {                                     // producer duty: keep the ring filled
+                if (lane == 0 && !produce(ti)) ok = false;
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+            }
+            const int stage = ti % S;
+            if (!warp_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
+            const int u0 = ti * U;
+          for (int ul = (kw + kKWarps - u0 % kKWarps) % kKWarps; ul < U; ul += kKWarps) {
+            const int u = u0 + ul;
+            const int ux = ul * 8;
+            const unsigned char* sK = smem + (size_t)stage * L.stage_bytes;
+            const unsigned char* sQ = sK + 2 * L.halo_pad;
+            // q of the lane's four pixels (rows 0..3 of column ux + g)
+            uint32_t qf[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = lds_u4(sQ, (uint32_t)(i * P.TW + ux + g) * 64u + tig * 16u);
+                qf[i][0] = v.x; qf[i][1] = v.y; qf[i][2] = v.z; qf[i][3] = v.w;
+            }
+            const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
+
+            float acc[2][3][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < 3; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+
+#pragma unroll
+            for (int dx = 0; dx < 3; ++dx) {
+                uint4 kc[6];                                       // one halo column, rows 0..5
+#pragma unroll
+                for (int r = 0; r < 6; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)(r * HW2 + dx) * 64u);
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy) {
+                        const int t = dy * 3 + dx;
+                        const uint4 k0 = kc[2 * mt + dy], k1 = kc[2 * mt + dy + 1];   // pixel rows 2mt / 2mt+1
+                        uint32_t a0[4], a1[4];
+                        a0[0] = hmul2_bf16(qf[2 * mt][0], k0.x);  a0[1] = hmul2_bf16(qf[2 * mt + 1][0], k1.x);
+                        a0[2] = hmul2_bf16(qf[2 * mt][1], k0.y);  a0[3] = hmul2_bf16(qf[2 * mt + 1][1], k1.y);
+                        a1[0] = hmul2_bf16(qf[2 * mt][2], k0.z);  a1[1] = hmul2_bf16(qf[2 * mt + 1][2], k1.z);
+                        a1[2] = hmul2_bf16(qf[2 * mt][3], k0.w);  a1[3] = hmul2_bf16(qf[2 * mt + 1][3], k1.w);
+                        mma_bf16(acc[mt][0], a0, bk[t][0][0], bk[t][0][1]);
+                        mma_bf16(acc[mt][1], a0, bk[t][0][2], bk[t][0][3]);
+                        mma_bf16(acc[mt][0], a1, bk[t][1][0], bk[t][1][1]);
+                        mma_bf16(acc[mt][1], a1, bk[t][1][2], bk[t][1][3]);
+                        if (t == 1) { mma_bf16(acc[mt][2], a0, ones_t1, ones_t1); mma_bf16(acc[mt][2], a1, ones_t1, ones_t1); }
+                        if (t == 8) { mma_bf16(acc[mt][2], a0, ones_t8, ones_t8); mma_bf16(acc[mt][2], a1, ones_t8, ones_t8); }
+                    }
+                }
+            }
+
+            // unnormalised softmax weights; the 4 lanes of a quad share a pixel
+            float e0[4], e1[4], e8[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int mt = i >> 1, o = (i & 1) * 2;
+                const float x0 = acc[mt][0][o], x1 = acc[mt][0][o + 1];
+                const float y0_ = acc[mt][1][o], y1_ = acc[mt][1][o + 1];
+                const float z0 = acc[mt][2][o], z1 = acc[mt][2][o + 1];
+                float l0, l1, l8;
+                if (tig == 0) { l0 = x0 + y1_; l1 = x1 + z0; l8 = (y0_ + z1) * P.scale_log2e + bias8; }
+                else          { l0 = x0 + y0_; l1 = x1 + y1_; l8 = -INFINITY; }
+                l0 = l0 * P.scale_log2e + bias0;
+                l1 = l1 * P.scale_log2e + bias1;
+                float m = fmaxf(fmaxf(l0, l1), l8);
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+                e0[i] = fast_exp2(l0 - m);
+                e1[i] = fast_exp2(l1 - m);
+                e8[i] = fast_exp2(l8 - m);
+            }
+
+            // rows of the block's A tile: pixel i of column g is row 32*quadrant + 8*i + g
+            const int blk = u >> 2, qd = u & 3, ab = blk % kABufs;
+            if (!warp_wait(bar(kBarAFree + ab), ((blk / kABufs) & 1) ^ 1)) { ok = false; break; }
+            unsigned char* sA = smem + L.a_off + ab * kABytes;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                unsigned char* row = sA + (4 * qd + i) * 512 + g * 16;
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(e0[i]), h1 = __float2bfloat16_rn(e1[i]);
+                const uint32_t hi = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+                const uint32_t lo = pack_bf16(e0[i] - __bfloat162float(h0), e1[i] - __bfloat162float(h1));
+                *reinterpret_cast<uint32_t*>(row + tig * 4) = hi;            // k 0..7   : meets D_v
+                *reinterpret_cast<uint32_t*>(row + 128 + tig * 4) = hi;      // k 8..15  : meets [s == t]
+                *reinterpret_cast<uint32_t*>(row + 256 + tig * 4) = lo;      // k 16..23 : meets [s == t]
+                if (tig == 0) {
+                    const __nv_bfloat16 h8 = __float2bfloat16_rn(e8[i]);
+                    const float f8 = __bfloat162float(h8);
+                    *reinterpret_cast<uint2*>(row + 384) = make_uint2(pack_bf16(f8, f8), pack_bf16(e8[i] - f8, 0.f));
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarAReady + ab));
+          }
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
+        }
+    } else if (warp < kVWarps) {
+        // =====================================================================================
+        // value warps (warp index = quadrant of the block = TMEM lanes 32*warp ..)
+        // =====================================================================================
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
+        const uint32_t tq = tmem + ((uint32_t)(32 * warp) << 16);
+
+        for (int ti = 0; ok && ti < my_tiles; ++ti) {
+            const int gt = rank + ti * nrank;
+            const int tx = gt % P.tiles_x;
+            const int ty = (gt / P.tiles_x) % P.tiles_y;
+            const int b = gt / (P.tiles_x * P.tiles_y);
+            const int stage = ti % S;
+            if (!warp_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
+            const int u0 = ti * U;
+          for (int ul = (warp + kVWarps - u0 % kVWarps) % kVWarps; ul < U; ul += kVWarps) {
+            const int u = u0 + ul;
+            const int ux = ul * 8;
+            const int blk = u >> 2;
+            const int r1 = (blk & 1) ? 2 : 0;                      // region of part 1
+            const uint32_t col1 = (blk & 1) ? kColP1b : kColP1a;
+            const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
+            const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
+
+            float o_acc[4][8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) o_acc[i][c] = 0.f;
+
+            if (!warp_wait(bar(kBarDFull + r1), (blk >> 1) & 1)) { ok = false; break; }
+            tc_fence_after_sync();
+#pragma unroll
+            for (int dx = 0; dx < 3; ++dx) {
+                if (dx == 2) {
+                    // part 1 is consumed; part 2 (taps with dx = 2, and the sums) comes next
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarDFree + r1));
+                    if (!warp_wait(bar(kBarDFull + 1), blk & 1)) { ok = false; break; }
+                    tc_fence_after_sync();
+                }
+                // one halo column of the strip, rows 0..5, widened to fp32 once
+                float vf[6][8];
+#pragma unroll
+                for (int r = 0; r < 6; ++r) {
+                    const uint4 v = lds_u4(sV, off0 + (uint32_t)(r * HW2 + dx) * 64u);
+                    vf[r][0] = bf16_lo(v.x); vf[r][1] = bf16_hi(v.x);
+                    vf[r][2] = bf16_lo(v.y); vf[r][3] = bf16_hi(v.y);
+                    vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
+                    vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
+                }
+                const uint32_t colbase = dx < 2 ? col1 + dx * 96 : kColP2;
+#pragma unroll
+                for (int r = 0; r < 5; ++r) {                      // rows r (half 0) and r+1 (half 1)
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        const int dy = r - 2 * mt;
+                        if (dy < 0 || dy > 2) continue;
+                        float d[16];                               // A'[pixel rows 2mt, 2mt+1][tap (dy,dx)][8 channels]
+                        tmem_ld_16x256b_x4(tq + ((uint32_t)(16 * mt) << 16) + colbase + dy * 32, d);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            ffma2(o_acc[2 * mt][2 * j], o_acc[2 * mt][2 * j + 1], d[4 * j], d[4 * j + 1],
+                                  vf[r][2 * j], vf[r][2 * j + 1]);
+                            ffma2(o_acc[2 * mt + 1][2 * j], o_acc[2 * mt + 1][2 * j + 1], d[4 * j + 2], d[4 * j + 3],
+                                  vf[r + 1][2 * j], vf[r + 1][2 * j + 1]);
+                        }
+                    }
+                }
+            }
+            if (!ok) break;
+            float inv[4];
+            {
+                float s0[4], s1[4];
+                tmem_ld_16x256b_x1(tq + kColP2 + 96, s0);                      // pixel rows 0, 1
+                tmem_ld_16x256b_x1(tq + (16u << 16) + kColP2 + 96, s1);        // pixel rows 2, 3
+                inv[0] = 1.f / s0[0]; inv[1] = 1.f / s0[2]; inv[2] = 1.f / s1[0]; inv[3] = 1.f / s1[2];
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarDFree + 1));
+
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int y = ty * 4 + i, x = tx * P.TW + ux + g;
+                if (y < P.H && x < P.W) {
+                    uint4 r;
+                    r.x = pack_bf16(o_acc[i][0] * inv[i], o_acc[i][1] * inv[i]);
+                    r.y = pack_bf16(o_acc[i][2] * inv[i], o_acc[i][3] * inv[i]);
+                    r.z = pack_bf16(o_acc[i][4] * inv[i], o_acc[i][5] * inv[i]);
+                    r.w = pack_bf16(o_acc[i][6] * inv[i], o_acc[i][7] * inv[i]);
+                    *reinterpret_cast<uint4*>(P.out + ((size_t)(b * P.H + y) * P.W + x) * C + h * kHeadDim + tig * 8) = r;
+                }
+            }
+          }
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
+        }
+        // quadrants of the last block that hold no unit: keep the region barriers in step
+        if (ok && my_blocks > 0 && (my_units & 3) != 0 && warp >= (my_units & 3)) {
+            const int blk = my_blocks - 1, r1 = (blk & 1) ? 2 : 0;
+            if (warp_wait(bar(kBarDFull + r1), (blk >> 1) & 1) && warp_wait(bar(kBarDFull + 1), blk & 1)) {
+                if (lane == 0) { mbar_arrive(bar(kBarDFree + r1)); mbar_arrive(bar(kBarDFree + 1)); }
+            } else {
+                ok = false;
+            }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kBarVDone));
+    } else {
+        // =====================================================================================
+        // control warp: lane 0 issues the value-side MMAs; the warp owns tensor memory
+        // =====================================================================================
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
+        if (lane == 0 && ok) {
+            ok = mbar_wait(bar(kBarWeightsDone), 0);               // B tile complete (and fenced)
+            const uint32_t sA0 = smem_u32(smem + L.a_off), sB0 = smem_u32(smem + L.b_off);
+            for (int blk = 0; ok && blk < my_blocks; ++blk) {
+                const int ab = blk % kABufs;
+                const int nunits = my_units - 4 * blk;             // the last block may be partial
+                for (int m = nunits; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
+                if (!mbar_wait(bar(kBarAReady + ab), (blk / kABufs) & 1)) { ok = false; break; }
+                const int r1 = (blk & 1) ? 2 : 0;
+                const uint32_t col1 = (blk & 1) ? kColP1b : kColP1a;
+                if (!mbar_wait(bar(kBarDFree + r1), ((blk >> 1) & 1) ^ 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t sA = sA0 + ab * kABytes;
+                // K = 32 = two instructions of K = 16 (two 8-element core matrices = 256 bytes each)
+                umma_bf16_ss(tmem + col1, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB0, 128, 512), kIdescP1, 0);
+                umma_bf16_ss(tmem + col1, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB0 + 256, 128, 512), kIdescP1, 1);
+                umma_commit(bar(kBarDFull + r1));
+                if (!mbar_wait(bar(kBarDFree + 1), (blk & 1) ^ 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t sB2 = sB0 + 24 * 512;               // column 192 onwards
+                umma_bf16_ss(tmem + kColP2, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB2, 128, 512), kIdescP2, 0);
+                umma_bf16_ss(tmem + kColP2, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB2 + 256, 128, 512), kIdescP2, 1);
+                umma_commit(bar(kBarDFull + 1));
+                umma_commit(bar(kBarAFree + ab));
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        // tensor memory is released once the value warps have stopped reading it (or given up)
+        if (my_tiles > 0 && !warp_wait(bar(kBarVDone), 0)) ok = false;
+        tc_fence_after_sync();
+        __syncwarp();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+    if (!ok && my_tiles > 0 && lane == 0) atomicExch(P.status, 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [B][H][W][C] bf16 as a 4-D tensor (C, W, H, B); box = 32 channels x bw pixels x bh rows x 1 image.
+bool make_map(CUtensorMap* map, const void* base, int B, int H, int W, int C, int bw, int bh) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)bw, (cuuint32_t)bh, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t kMaxSmem = 227 * 1024;
+
+}  // namespace
+
+bool umma_supports(slide_attn_dtype dtype, int head_dim, int ksize) {
+    return dtype == SLIDE_ATTN_BF16 && head_dim == kHeadDim && ksize == 3;
+}
+
+cudaError_t umma_setup() {
+    if (!encode_fn()) return cudaErrorNotSupported;
+    return cudaFuncSetAttribute(umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+}
+
+cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream_t stream) {
+    // tile width: a multiple of 8 up to 64, splitting the row evenly
+    const int txn = (p.W + 63) / 64;
+    const int TW = ((((p.W + txn - 1) / txn) + 7) / 8) * 8;
+    UmmaParams P;
+    P.wk = p.wk; P.wv = p.wv; P.bias = p.bias;
+    P.out = static_cast<__nv_bfloat16*>(p.out);
+    P.status = d_status;
+    P.B = p.B; P.H = p.H; P.W = p.W; P.heads = p.heads;
+    P.TW = TW;
+    P.tiles_x = (p.W + TW - 1) / TW;
+    P.tiles_y = (p.H + 3) / 4;
+    P.stages = smem_layout(TW, 3).total <= kMaxSmem ? 3 : 2;
+    P.scale_log2e = kLog2e / sqrtf((float)kHeadDim);
+    const Smem L = smem_layout(TW, P.stages);
+    if (L.total > kMaxSmem) return cudaErrorInvalidConfiguration;
+
+    const int C = p.heads * kHeadDim;
+    CUtensorMap map_q, map_k, map_v;
+    if (!make_map(&map_q, p.q, p.B, p.H, p.W, C, TW, 4) ||
+        !make_map(&map_k, p.k, p.B, p.H, p.W, C, TW + 2, 6) ||
+        !make_map(&map_v, p.v, p.B, p.H, p.W, C, TW + 2, 6))
+        return cudaErrorInvalidValue;
+
+    const long long tiles = (long long)P.tiles_x * P.tiles_y * p.B * p.heads;
+    if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    int grid = num_sms;
+    if (grid < p.heads) grid = p.heads;                    // every head needs at least one CTA
+    if ((long long)grid > tiles) grid = (int)tiles;
+    umma_kernel<<<grid, kThreads, L.total, stream>>>(map_q, map_k, map_v, P);
+    return cudaGetLastError();
+}
+
+}  // namespace slide_attn

@@ -27,15 +27,17 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
-// Bounded wait: false if the phase did not complete within the spin limit.
+// Bounded wait: false if the phase did not complete within the limit (about two seconds).  Each
+// probe may park the thread for up to 100 us (the hardware wakes it when the phase completes), so
+// a waiting warp issues next to no instructions.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int spin = 0; spin < (1 << 20); ++spin) {
+    for (int spin = 0; spin < 20000; ++spin) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+            : "=r"(done) : "r"(bar), "r"(parity), "r"(100000u) : "memory");
         if (done) return true;
     }
     return false;

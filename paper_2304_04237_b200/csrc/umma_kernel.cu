@@ -17,11 +17,11 @@
 //   B column (t,c) (shared memory, built once per CTA):  D_v[c][0..7][t] | [s == t] | [s == t] |
 //                                                       D_v[c][8][t], [t == 8], [t == 8], 0 ...
 //   16 more columns hold 0 | 1 | 1 | 0,1,1,0... and so deliver sum_s e[p,s].
-// D (fp32) lives in tensor memory, pixel = TMEM lane.  Columns are ordered by tap column dx: the
-// taps with dx = 0, 1 (192 columns) form part 1, those with dx = 2 plus the sum columns (112) part
-// 2.  Part 1 is double-buffered across blocks, part 2 single-buffered (192 + 112 + 192 = 496 of the
-// 512 TMEM columns).  Value warp w reads TMEM lanes 32w .. 32w+31 (its quadrant) with
-// tcgen05.ld.16x256b, whose register layout equals the mma.sync accumulator fragment.
+// D (fp32) lives in tensor memory, pixel = TMEM lane.  Columns are ordered by tap column dx; the
+// three taps of one dx (96 columns; the last dx also carries the 16 sum columns) form a chunk, and
+// chunks go round a ring of four 112-column TMEM slots, so the MMA of a chunk is issued about one
+// block ahead of the value warps that read it.  Value warp w reads TMEM lanes 32w .. 32w+31 (its
+// quadrant) with tcgen05.ld.16x256b, whose register layout equals the mma.sync accumulator fragment.
 //
 // Roles (12 warps): warps 0-3 value warps (warp index = TMEM quadrant = unit index within a block),
 // warps 4-10 key warps (lane 0 of the first one is the TMA producer), warp 11 allocates / frees
@@ -47,9 +47,10 @@ constexpr int kBBytes = kBCols * 64;
 constexpr int kWeightBytes = kHeadDim * 81 * 4;         // fp32 weights of one head, one side
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColP1a = 0, kColP2 = 192, kColP1b = 304;   // TMEM column regions
-constexpr uint32_t kIdescP1 = umma_idesc_bf16(128, 192);
-constexpr uint32_t kIdescP2 = umma_idesc_bf16(128, 112);
+constexpr int kDSlots = 4;                              // ring of TMEM chunks
+constexpr uint32_t kDSlotCols = 112;
+constexpr uint32_t kIdesc96 = umma_idesc_bf16(128, 96);
+constexpr uint32_t kIdesc112 = umma_idesc_bf16(128, 112);
 
 struct UmmaParams {
     const float* wk;
@@ -96,9 +97,9 @@ constexpr int kBarWeights = 6;       // weights landed
 constexpr int kBarWeightsDone = 7;   // all warps have built their fragments / their share of the B tile
 constexpr int kBarAReady = 8;        // [A buffer]  the 4 units of a block have written their rows
 constexpr int kBarAFree = 11;        // [A buffer]  the MMAs reading the buffer are complete
-constexpr int kBarDFull = 14;        // [region: part 1 even, part 2, part 1 odd]  MMA results in TMEM
-constexpr int kBarDFree = 17;        // [region]  the 4 value warps are done reading the region
-constexpr int kBarVDone = 20;        // value warps have finished all TMEM reads
+constexpr int kBarDFull = 14;        // [TMEM slot]  MMA results of a chunk are in tensor memory
+constexpr int kBarDFree = 18;        // [TMEM slot]  the 4 value warps are done reading the chunk
+constexpr int kBarVDone = 22;        // value warps have finished all TMEM reads
 
 __device__ __forceinline__ float4 lds_f4(const unsigned char* base, uint32_t off) {
     return *reinterpret_cast<const float4*>(base + off);
@@ -163,7 +164,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             mbar_init(bar(kBarAReady + i), 4);
             mbar_init(bar(kBarAFree + i), 1);
         }
-        for (int i = 0; i < 3; ++i) {
+        for (int i = 0; i < kDSlots; ++i) {
             mbar_init(bar(kBarDFull + i), 1);
             mbar_init(bar(kBarDFree + i), kVWarps);
         }
@@ -403,8 +404,6 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             const int u = u0 + ul;
             const int ux = ul * 8;
             const int blk = u >> 2;
-            const int r1 = (blk & 1) ? 2 : 0;                      // region of part 1
-            const uint32_t col1 = (blk & 1) ? kColP1b : kColP1a;
             const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
             const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
 
@@ -413,19 +412,13 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int c = 0; c < 8; ++c) o_acc[i][c] = 0.f;
+            float inv[4] = {0.f, 0.f, 0.f, 0.f};
 
-            if (!warp_wait(bar(kBarDFull + r1), (blk >> 1) & 1)) { ok = false; break; }
-            tc_fence_after_sync();
 #pragma unroll
             for (int dx = 0; dx < 3; ++dx) {
-                if (dx == 2) {
-                    // part 1 is consumed; part 2 (taps with dx = 2, and the sums) comes next
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(kBarDFree + r1));
-                    if (!warp_wait(bar(kBarDFull + 1), blk & 1)) { ok = false; break; }
-                    tc_fence_after_sync();
-                }
+                const int ci = 3 * blk + dx, ds = ci % kDSlots;       // chunk index and its TMEM slot
+                if (!warp_wait(bar(kBarDFull + ds), (ci / kDSlots) & 1)) { ok = false; break; }
+                tc_fence_after_sync();
                 // one halo column of the strip, rows 0..5, widened to fp32 once
                 float vf[6][8];
 #pragma unroll
@@ -436,7 +429,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
                     vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
                 }
-                const uint32_t colbase = dx < 2 ? col1 + dx * 96 : kColP2;
+                const uint32_t colbase = ds * kDSlotCols;
 #pragma unroll
                 for (int r = 0; r < 5; ++r) {                      // rows r (half 0) and r+1 (half 1)
 #pragma unroll
@@ -454,18 +447,17 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                         }
                     }
                 }
+                if (dx == 2) {                                     // sum_s e[p,s] of the four pixels
+                    float s0[4], s1[4];
+                    tmem_ld_16x256b_x1(tq + colbase + 96, s0);                      // pixel rows 0, 1
+                    tmem_ld_16x256b_x1(tq + (16u << 16) + colbase + 96, s1);        // pixel rows 2, 3
+                    inv[0] = 1.f / s0[0]; inv[1] = 1.f / s0[2]; inv[2] = 1.f / s1[0]; inv[3] = 1.f / s1[2];
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
             }
             if (!ok) break;
-            float inv[4];
-            {
-                float s0[4], s1[4];
-                tmem_ld_16x256b_x1(tq + kColP2 + 96, s0);                      // pixel rows 0, 1
-                tmem_ld_16x256b_x1(tq + (16u << 16) + kColP2 + 96, s1);        // pixel rows 2, 3
-                inv[0] = 1.f / s0[0]; inv[1] = 1.f / s0[2]; inv[2] = 1.f / s1[0]; inv[3] = 1.f / s1[2];
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarDFree + 1));
 
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -483,13 +475,12 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             __syncwarp();
             if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
         }
-        // quadrants of the last block that hold no unit: keep the region barriers in step
+        // quadrants of the last block that hold no unit: keep the chunk barriers in step
         if (ok && my_blocks > 0 && (my_units & 3) != 0 && warp >= (my_units & 3)) {
-            const int blk = my_blocks - 1, r1 = (blk & 1) ? 2 : 0;
-            if (warp_wait(bar(kBarDFull + r1), (blk >> 1) & 1) && warp_wait(bar(kBarDFull + 1), blk & 1)) {
-                if (lane == 0) { mbar_arrive(bar(kBarDFree + r1)); mbar_arrive(bar(kBarDFree + 1)); }
-            } else {
-                ok = false;
+            for (int dx = 0; ok && dx < 3; ++dx) {
+                const int ci = 3 * (my_blocks - 1) + dx, ds = ci % kDSlots;
+                if (!warp_wait(bar(kBarDFull + ds), (ci / kDSlots) & 1)) { ok = false; break; }
+                if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
             }
         }
         tc_fence_before_sync();
@@ -509,21 +500,20 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 const int nunits = my_units - 4 * blk;             // the last block may be partial
                 for (int m = nunits; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
                 if (!mbar_wait(bar(kBarAReady + ab), (blk / kABufs) & 1)) { ok = false; break; }
-                const int r1 = (blk & 1) ? 2 : 0;
-                const uint32_t col1 = (blk & 1) ? kColP1b : kColP1a;
-                if (!mbar_wait(bar(kBarDFree + r1), ((blk >> 1) & 1) ^ 1)) { ok = false; break; }
-                tc_fence_after_sync();
                 const uint32_t sA = sA0 + ab * kABytes;
-                // K = 32 = two instructions of K = 16 (two 8-element core matrices = 256 bytes each)
-                umma_bf16_ss(tmem + col1, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB0, 128, 512), kIdescP1, 0);
-                umma_bf16_ss(tmem + col1, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB0 + 256, 128, 512), kIdescP1, 1);
-                umma_commit(bar(kBarDFull + r1));
-                if (!mbar_wait(bar(kBarDFree + 1), (blk & 1) ^ 1)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t sB2 = sB0 + 24 * 512;               // column 192 onwards
-                umma_bf16_ss(tmem + kColP2, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB2, 128, 512), kIdescP2, 0);
-                umma_bf16_ss(tmem + kColP2, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB2 + 256, 128, 512), kIdescP2, 1);
-                umma_commit(bar(kBarDFull + 1));
+                for (int dx = 0; dx < 3; ++dx) {
+                    const int ci = 3 * blk + dx, ds = ci % kDSlots;
+                    if (!mbar_wait(bar(kBarDFree + ds), ((ci / kDSlots) & 1) ^ 1)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    // columns dx*96 .. of B; K = 32 = two instructions of K = 16 (256 bytes apart)
+                    const uint32_t sB = sB0 + dx * 12 * 512;
+                    const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
+                    const uint32_t dcol = tmem + ds * kDSlotCols;
+                    umma_bf16_ss(dcol, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB, 128, 512), idesc, 0);
+                    umma_bf16_ss(dcol, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB + 256, 128, 512), idesc, 1);
+                    umma_commit(bar(kBarDFull + ds));
+                }
+                if (!ok) break;
                 umma_commit(bar(kBarAFree + ab));
             }
         }

@@ -24,8 +24,8 @@
 // quadrant) with tcgen05.ld.16x256b, whose register layout equals the mma.sync accumulator fragment.
 //
 // Roles (12 warps): warps 0-3 value warps (warp index = TMEM quadrant = unit index within a block),
-// warps 4-10 key warps (lane 0 of the first one is the TMA producer), warp 11 allocates / frees
-// tensor memory and its lane 0 issues the MMAs.  Every wait is bounded; a wait that runs out sets
+// warps 4-10 key warps, warp 11 allocates / frees tensor memory and its lane 0 is the scheduler:
+// it issues the TMA loads and the MMAs.  Every wait is bounded; a wait that runs out sets
 // the status word, and tensor memory is released on every path.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -113,20 +113,6 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
 }
 
-// Value B(n, k) of the value-side MMA for one head; wv: fp32 [32][9][9] of the head.
-__device__ __forceinline__ float b_value(const float* wv, int n, int k) {
-    if (n >= 288) return (k >= 8 && k < 24) || k == 25 || k == 26 ? 1.f : 0.f;      // sum columns
-    const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;          // columns are ordered dx-major
-    const int cn = n & 31, j = cn >> 3, wi = cn & 7;
-    const int c = 8 * (wi >> 1) + 2 * j + (wi & 1);
-    if (k < 8) return wv[c * 81 + k * 9 + t] - (k == t ? 1.f : 0.f);
-    if (k < 16) return (k - 8) == t ? 1.f : 0.f;
-    if (k < 24) return (k - 16) == t ? 1.f : 0.f;
-    if (k == 24) return wv[c * 81 + 72 + t] - (t == 8 ? 1.f : 0.f);
-    if (k == 25 || k == 26) return t == 8 ? 1.f : 0.f;
-    return 0.f;
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
             const __grid_constant__ CUtensorMap map_v, const UmmaParams P)
@@ -197,31 +183,14 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     // The fp32 weights of the head are staged in the LAST stage's memory; that stage receives its
     // first tile only after every warp has finished with them.
     const unsigned char* w_stage = smem + (size_t)(S - 1) * L.stage_bytes;
-    int issued = 0;                                            // producer state (first key warp, lane 0)
-    if (my_tiles > 0 && warp == kVWarps && lane == 0) {
+    int issued = 0;                                            // producer state (control warp, lane 0)
+    if (my_tiles > 0 && warp == kCtlWarp && lane == 0) {
         mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
         bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
         bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
         while (issued < my_tiles && issued < S - 1) issue_tile(issued++);
     }
     __syncwarp();
-
-    // Issues every tile whose stage is free.  A tile that the producer's own warp needs now (index
-    // <= `need`) is waited for; later ones are only probed.  Returns false if a wait ran out.
-    auto produce = [&](int need) -> bool {
-        while (issued < my_tiles) {
-            uint32_t b = 0, par = 0;
-            bool gated = false;
-            if (issued == S - 1) { b = bar(kBarWeightsDone); par = 0; gated = true; }   // staging area must be dead
-            else if (issued >= S) { b = bar(kBarEmpty + issued % S); par = ((issued / S) - 1) & 1; gated = true; }
-            if (gated && !mbar_test(b, par)) {
-                if (issued > need) return true;               // not needed yet: try again later
-                if (!mbar_wait(b, par)) return false;
-            }
-            issue_tile(issued++);
-        }
-        return true;
-    };
 
     bool ok = my_tiles > 0 && warp_wait(bar(kBarWeights), 0);
     const float* wks = reinterpret_cast<const float*>(w_stage);
@@ -230,10 +199,32 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     // ---- B tile of the value-side MMA: every thread converts its share ---------------------------
     if (ok) {
         unsigned char* sB = smem + L.b_off;
-        for (int idx = threadIdx.x; idx < kBCols * 16; idx += kThreads) {
-            const int n = idx >> 4, k = (idx & 15) * 2;
-            const uint32_t w = pack_bf16(b_value(wvs, n, k), b_value(wvs, n, k + 1));
-            *reinterpret_cast<uint32_t*>(sB + (n >> 3) * 512 + (k >> 3) * 128 + (n & 7) * 16 + (k & 7) * 2) = w;
+        for (int n = threadIdx.x; n < kBCols; n += kThreads) {     // one column (64 bytes of K) per thread
+            unsigned char* col = sB + (n >> 3) * 512 + (n & 7) * 16;
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i] = 0u;
+            if (n >= 288) {                                         // sum columns: 0 | 1 | 1 | 0,1,1,0..
+#pragma unroll
+                for (int i = 4; i < 12; ++i) w[i] = kOnesBf16x2;
+                w[12] = pack_bf16(0.f, 1.f); w[13] = pack_bf16(1.f, 0.f);
+            } else {
+                const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;  // columns are ordered dx-major
+                const int cn = n & 31, j = cn >> 3, wi = cn & 7;
+                const float* wc = wvs + (8 * (wi >> 1) + 2 * j + (wi & 1)) * 81 + t;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int s0 = 2 * i, s1 = 2 * i + 1;
+                    w[i] = pack_bf16(wc[s0 * 9] - (s0 == t ? 1.f : 0.f), wc[s1 * 9] - (s1 == t ? 1.f : 0.f));
+                    const uint32_t oh = pack_bf16(s0 == t ? 1.f : 0.f, s1 == t ? 1.f : 0.f);
+                    w[4 + i] = oh; w[8 + i] = oh;
+                }
+                const float o8 = t == 8 ? 1.f : 0.f;
+                w[12] = pack_bf16(wc[72] - o8, o8); w[13] = pack_bf16(o8, 0.f);
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4*>(col + c * 128) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
         }
         fence_proxy_async_smem();
     }
@@ -281,11 +272,6 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         // a tile in which it owns no unit: a warp that skipped a phase of a barrier could later
         // mistake an older phase for the one it waits for.
         for (int ti = 0; ok && ti < my_tiles; ++ti) {
-            if (kw == 0) {                                     // producer duty: keep the ring filled
-                if (lane == 0 && !produce(ti)) ok = false;
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                if (!ok) break;
-            }
             const int stage = ti % S;
             if (!warp_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
             const int u0 = ti * U;
@@ -431,18 +417,19 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 }
                 const uint32_t colbase = ds * kDSlotCols;
 #pragma unroll
-                for (int r = 0; r < 5; ++r) {                      // rows r (half 0) and r+1 (half 1)
+                for (int mt = 0; mt < 2; ++mt) {
+                    // A'[pixel rows 2mt, 2mt+1][taps (dy = 0..2, dx)][8 channels]: three loads in flight
+                    float d[48];
+                    const uint32_t ta = tq + ((uint32_t)(16 * mt) << 16) + colbase;
+                    tmem_ld3_16x256b_x4(ta, ta + 32, ta + 64, d);
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        const int dy = r - 2 * mt;
-                        if (dy < 0 || dy > 2) continue;
-                        float d[16];                               // A'[pixel rows 2mt, 2mt+1][tap (dy,dx)][8 channels]
-                        tmem_ld_16x256b_x4(tq + ((uint32_t)(16 * mt) << 16) + colbase + dy * 32, d);
+                    for (int dy = 0; dy < 3; ++dy) {
+                        const int r = 2 * mt + dy;                 // halo rows r (half 0) and r+1 (half 1)
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            ffma2(o_acc[2 * mt][2 * j], o_acc[2 * mt][2 * j + 1], d[4 * j], d[4 * j + 1],
+                            ffma2(o_acc[2 * mt][2 * j], o_acc[2 * mt][2 * j + 1], d[16 * dy + 4 * j], d[16 * dy + 4 * j + 1],
                                   vf[r][2 * j], vf[r][2 * j + 1]);
-                            ffma2(o_acc[2 * mt + 1][2 * j], o_acc[2 * mt + 1][2 * j + 1], d[4 * j + 2], d[4 * j + 3],
+                            ffma2(o_acc[2 * mt + 1][2 * j], o_acc[2 * mt + 1][2 * j + 1], d[16 * dy + 4 * j + 2], d[16 * dy + 4 * j + 3],
                                   vf[r + 1][2 * j], vf[r + 1][2 * j + 1]);
                         }
                     }
@@ -459,16 +446,20 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             }
             if (!ok) break;
 
+            {
+                const int x = tx * P.TW + ux + g, y0 = ty * 4;
+                __nv_bfloat16* op = P.out + ((size_t)(b * P.H + y0) * P.W + x) * C + h * kHeadDim + tig * 8;
+                const size_t row_stride = (size_t)P.W * C;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int y = ty * 4 + i, x = tx * P.TW + ux + g;
-                if (y < P.H && x < P.W) {
-                    uint4 r;
-                    r.x = pack_bf16(o_acc[i][0] * inv[i], o_acc[i][1] * inv[i]);
-                    r.y = pack_bf16(o_acc[i][2] * inv[i], o_acc[i][3] * inv[i]);
-                    r.z = pack_bf16(o_acc[i][4] * inv[i], o_acc[i][5] * inv[i]);
-                    r.w = pack_bf16(o_acc[i][6] * inv[i], o_acc[i][7] * inv[i]);
-                    *reinterpret_cast<uint4*>(P.out + ((size_t)(b * P.H + y) * P.W + x) * C + h * kHeadDim + tig * 8) = r;
+                for (int i = 0; i < 4; ++i) {
+                    if (x < P.W && y0 + i < P.H) {
+                        uint4 r;
+                        r.x = pack_bf16(o_acc[i][0] * inv[i], o_acc[i][1] * inv[i]);
+                        r.y = pack_bf16(o_acc[i][2] * inv[i], o_acc[i][3] * inv[i]);
+                        r.z = pack_bf16(o_acc[i][4] * inv[i], o_acc[i][5] * inv[i]);
+                        r.w = pack_bf16(o_acc[i][6] * inv[i], o_acc[i][7] * inv[i]);
+                        *reinterpret_cast<uint4*>(op + i * row_stride) = r;
+                    }
                 }
             }
           }
@@ -493,28 +484,54 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
         if (lane == 0 && ok) {
-            ok = mbar_wait(bar(kBarWeightsDone), 0);               // B tile complete (and fenced)
+            // One thread runs both queues by polling, so neither can hold up the other:
+            //   TMA queue: tile n goes out as soon as its stage is free;
+            //   MMA queue: chunk (blk, dx) goes out as soon as the block's A tile is complete and
+            //   its TMEM slot has been read.
+            // It gives up when nothing has moved for about two seconds.
             const uint32_t sA0 = smem_u32(smem + L.a_off), sB0 = smem_u32(smem + L.b_off);
-            for (int blk = 0; ok && blk < my_blocks; ++blk) {
-                const int ab = blk % kABufs;
-                const int nunits = my_units - 4 * blk;             // the last block may be partial
-                for (int m = nunits; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
-                if (!mbar_wait(bar(kBarAReady + ab), (blk / kABufs) & 1)) { ok = false; break; }
-                const uint32_t sA = sA0 + ab * kABytes;
-                for (int dx = 0; dx < 3; ++dx) {
-                    const int ci = 3 * blk + dx, ds = ci % kDSlots;
-                    if (!mbar_wait(bar(kBarDFree + ds), ((ci / kDSlots) & 1) ^ 1)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    // columns dx*96 .. of B; K = 32 = two instructions of K = 16 (256 bytes apart)
-                    const uint32_t sB = sB0 + dx * 12 * 512;
-                    const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
-                    const uint32_t dcol = tmem + ds * kDSlotCols;
-                    umma_bf16_ss(dcol, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB, 128, 512), idesc, 0);
-                    umma_bf16_ss(dcol, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB + 256, 128, 512), idesc, 1);
-                    umma_commit(bar(kBarDFull + ds));
+            bool weights_done = false, a_ready = false;
+            int blk = 0, dx = 0;
+            long long last_progress = clock64();
+            while (issued < my_tiles || blk < my_blocks) {
+                bool progress = false;
+                if (!weights_done && mbar_test(bar(kBarWeightsDone), 0)) { weights_done = true; progress = true; }
+                if (issued < my_tiles) {
+                    bool free_now;
+                    if (issued < S - 1) free_now = true;
+                    else if (issued == S - 1) free_now = weights_done;          // staging area must be dead
+                    else free_now = mbar_test(bar(kBarEmpty + issued % S), ((issued / S) - 1) & 1);
+                    if (free_now) { issue_tile(issued++); progress = true; }
                 }
-                if (!ok) break;
-                umma_commit(bar(kBarAFree + ab));
+                if (blk < my_blocks && weights_done) {
+                    const int ab = blk % kABufs;
+                    if (dx == 0 && !a_ready) {
+                        if (blk == my_blocks - 1 && (my_units & 3) != 0) {       // partial last block: stand in
+                            for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
+                        }
+                        a_ready = true;                                          // now only the barrier decides
+                    }
+                    const int ci = 3 * blk + dx, ds = ci % kDSlots;
+                    if (mbar_test(bar(kBarAReady + ab), (blk / kABufs) & 1) &&
+                        mbar_test(bar(kBarDFree + ds), ((ci / kDSlots) & 1) ^ 1)) {
+                        tc_fence_after_sync();
+                        // columns dx*96 .. of B; K = 32 = two instructions of K = 16 (256 bytes apart)
+                        const uint32_t sA = sA0 + ab * kABytes, sB = sB0 + dx * 12 * 512;
+                        const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
+                        const uint32_t dcol = tmem + ds * kDSlotCols;
+                        umma_bf16_ss(dcol, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB, 128, 512), idesc, 0);
+                        umma_bf16_ss(dcol, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB + 256, 128, 512), idesc, 1);
+                        umma_commit(bar(kBarDFull + ds));
+                        if (++dx == 3) { umma_commit(bar(kBarAFree + ab)); dx = 0; ++blk; a_ready = false; }
+                        progress = true;
+                    }
+                }
+                if (progress) {
+                    last_progress = clock64();
+                } else {
+                    if (clock64() - last_progress > 4000000000LL) { ok = false; break; }
+                    __nanosleep(40);
+                }
             }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;

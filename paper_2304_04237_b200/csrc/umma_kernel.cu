@@ -23,9 +23,10 @@
 // block ahead of the value warps that read it.  Value warp w reads TMEM lanes 32w .. 32w+31 (its
 // quadrant) with tcgen05.ld.16x256b, whose register layout equals the mma.sync accumulator fragment.
 //
-// Roles (12 warps): warps 0-3 value warps (warp index = TMEM quadrant = unit index within a block),
-// warps 4-10 key warps, warp 11 allocates / frees tensor memory and its lane 0 is the scheduler:
-// it issues the TMA loads and the MMAs.  Every wait is bounded; a wait that runs out sets
+// Roles (16 warps, 128 registers each): warps 0-7 value warps (warp % 4 = TMEM quadrant = unit index
+// within a block; warps w and w+4 take alternate blocks), warps 8-14 key warps (their B fragments
+// are re-read from shared memory for every unit), warp 15 allocates / frees tensor memory and its
+// lane 0 is the scheduler: it issues the TMA loads and the MMAs.  Every wait is bounded; a wait that runs out sets
 // the status word, and tensor memory is released on every path.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -35,12 +36,13 @@ namespace slide_attn {
 namespace {
 
 constexpr int kHeadDim = 32;
-constexpr int kVWarps = 4;
+constexpr int kVWarps = 8;
 constexpr int kKWarps = 7;
-constexpr int kCtlWarp = kVWarps + kKWarps;             // warp 11
+constexpr int kCtlWarp = kVWarps + kKWarps;             // warp 15
 constexpr int kThreads = (kVWarps + kKWarps + 1) * 32;
 constexpr int kMaxStages = 3;
-constexpr int kABufs = 3;                               // A tiles (one per block in flight)
+constexpr int kABufs = 2;                               // A tiles (one per block in flight)
+constexpr int kBkBytes = 9 * 2 * 32 * 16;               // key-side B fragments of the head, fragment order
 constexpr int kABytes = 128 * 64;                       // 128 rows x 32 bf16
 constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
 constexpr int kBBytes = kBCols * 64;
@@ -69,6 +71,7 @@ struct Smem {
     uint32_t halo_pad;         // bytes of one K or V halo tile (6 rows x (TW+2) pixels x 64 B), 1024-aligned
     uint32_t stage_bytes;      // K halo | V halo | q tile
     uint32_t b_off;            // B tile of the value-side MMA
+    uint32_t bk_off;           // key-side B fragments [tap][k-step][lane][4 words]
     uint32_t a_off;            // A tiles [kABufs][kABytes]
     uint32_t tmem_off;         // TMEM base address written by tcgen05.alloc
     uint32_t bar_off;          // mbarriers
@@ -83,7 +86,8 @@ __host__ __device__ inline Smem smem_layout(int TW, int stages) {
     const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
     if (s.stage_bytes < wbytes) s.stage_bytes = wbytes;
     s.b_off = s.stage_bytes * stages;
-    s.a_off = s.b_off + kBBytes;
+    s.bk_off = s.b_off + kBBytes;
+    s.a_off = s.bk_off + kBkBytes;
     s.tmem_off = s.a_off + kABufs * kABytes;
     s.bar_off = s.tmem_off + 16;
     s.total = s.bar_off + 32 * 8 + 1024;
@@ -152,7 +156,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         }
         for (int i = 0; i < kDSlots; ++i) {
             mbar_init(bar(kBarDFull + i), 1);
-            mbar_init(bar(kBarDFree + i), kVWarps);
+            mbar_init(bar(kBarDFree + i), 4);
         }
         mbar_init(bar(kBarVDone), kVWarps);
     }
@@ -226,35 +230,32 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             for (int c = 0; c < 4; ++c)
                 *reinterpret_cast<uint4*>(col + c * 128) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
         }
+        // key-side B fragments in fragment order: word (t, ks, lane, i) with n-tile i/2, register i%2
+        uint32_t* sBk = reinterpret_cast<uint32_t*>(smem + L.bk_off);
+        for (int w = threadIdx.x; w < 9 * 2 * 32 * 4; w += kThreads) {
+            const int i = w & 3, ln = (w >> 2) & 31, ks = (w >> 7) & 1, t = w >> 8;
+            const int fg = ln >> 2, ft = ln & 3, r = i & 1;
+            const int c0 = 8 * ft + 4 * ks + 2 * r;
+            uint32_t word;
+            if ((i >> 1) == 0 || fg == 0) {                        // n-tile 0: slot fg; n-tile 1 column 0: slot 8
+                const int sl = (i >> 1) == 0 ? fg : 8;
+                const float e = (sl == t) ? 1.f : 0.f;
+                word = pack_bf16(wks[c0 * 81 + sl * 9 + t] - e, wks[(c0 + 1) * 81 + sl * 9 + t] - e);
+            } else {                                               // n-tile 1: column 1 sums tap 0, column n >= 2 tap n
+                word = t == (fg == 1 ? 0 : fg) ? kOnesBf16x2 : 0u;
+            }
+            sBk[w] = word;
+        }
         fence_proxy_async_smem();
     }
+    __syncthreads();                                               // B tile and key-side fragments are complete
 
     if (warp >= kVWarps && warp < kCtlWarp) {
         // =====================================================================================
         // key warps
         // =====================================================================================
         const int kw = warp - kVWarps;
-        uint32_t bk[9][2][4];          // [tap][k-step][n-tile 0: r0 r1 | n-tile 1: r0 r1]
-        if (ok) {
-#pragma unroll
-            for (int t = 0; t < 9; ++t)
-#pragma unroll
-                for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        const int c0 = 8 * tig + 4 * ks + 2 * r;
-                        {   // n-tile 0: column g = slot g
-                            const float e = (g == t) ? 1.f : 0.f;
-                            bk[t][ks][r] = pack_bf16(wks[c0 * 81 + g * 9 + t] - e, wks[(c0 + 1) * 81 + g * 9 + t] - e);
-                        }
-                        {   // n-tile 1: column 0 = slot 8; column 1 sums tap 0; column n >= 2 sums tap n
-                            const float e = (t == 8) ? 1.f : 0.f;
-                            const uint32_t d = pack_bf16(wks[c0 * 81 + 72 + t] - e, wks[(c0 + 1) * 81 + 72 + t] - e);
-                            const int tap = g == 1 ? 0 : g;
-                            bk[t][ks][2 + r] = g == 0 ? d : (t == tap ? kOnesBf16x2 : 0u);
-                        }
-                    }
-        }
+        const unsigned char* sBk = smem + L.bk_off + lane * 16;
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
 
@@ -303,20 +304,21 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
 #pragma unroll
                 for (int r = 0; r < 6; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)(r * HW2 + dx) * 64u);
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
+                for (int dy = 0; dy < 3; ++dy) {
+                    const int t = dy * 3 + dx;
+                    const uint4 b0 = lds_u4(sBk, (t * 2 + 0) * 512), b1 = lds_u4(sBk, (t * 2 + 1) * 512);
 #pragma unroll
-                    for (int dy = 0; dy < 3; ++dy) {
-                        const int t = dy * 3 + dx;
+                    for (int mt = 0; mt < 2; ++mt) {
                         const uint4 k0 = kc[2 * mt + dy], k1 = kc[2 * mt + dy + 1];   // pixel rows 2mt / 2mt+1
                         uint32_t a0[4], a1[4];
                         a0[0] = hmul2_bf16(qf[2 * mt][0], k0.x);  a0[1] = hmul2_bf16(qf[2 * mt + 1][0], k1.x);
                         a0[2] = hmul2_bf16(qf[2 * mt][1], k0.y);  a0[3] = hmul2_bf16(qf[2 * mt + 1][1], k1.y);
                         a1[0] = hmul2_bf16(qf[2 * mt][2], k0.z);  a1[1] = hmul2_bf16(qf[2 * mt + 1][2], k1.z);
                         a1[2] = hmul2_bf16(qf[2 * mt][3], k0.w);  a1[3] = hmul2_bf16(qf[2 * mt + 1][3], k1.w);
-                        mma_bf16(acc[mt][0], a0, bk[t][0][0], bk[t][0][1]);
-                        mma_bf16(acc[mt][1], a0, bk[t][0][2], bk[t][0][3]);
-                        mma_bf16(acc[mt][0], a1, bk[t][1][0], bk[t][1][1]);
-                        mma_bf16(acc[mt][1], a1, bk[t][1][2], bk[t][1][3]);
+                        mma_bf16(acc[mt][0], a0, b0.x, b0.y);
+                        mma_bf16(acc[mt][1], a0, b0.z, b0.w);
+                        mma_bf16(acc[mt][0], a1, b1.x, b1.y);
+                        mma_bf16(acc[mt][1], a1, b1.z, b1.w);
                         if (t == 1) { mma_bf16(acc[mt][2], a0, ones_t1, ones_t1); mma_bf16(acc[mt][2], a1, ones_t1, ones_t1); }
                         if (t == 8) { mma_bf16(acc[mt][2], a0, ones_t8, ones_t8); mma_bf16(acc[mt][2], a1, ones_t8, ones_t8); }
                     }
@@ -376,7 +378,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         // =====================================================================================
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
-        const uint32_t tq = tmem + ((uint32_t)(32 * warp) << 16);
+        const int qd = warp & 3, half = warp >> 2;                 // quadrant; which blocks (even / odd)
+        const uint32_t tq = tmem + ((uint32_t)(32 * qd) << 16);
 
         for (int ti = 0; ok && ti < my_tiles; ++ti) {
             const int gt = rank + ti * nrank;
@@ -386,8 +389,9 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             const int stage = ti % S;
             if (!warp_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
             const int u0 = ti * U;
-          for (int ul = (warp + kVWarps - u0 % kVWarps) % kVWarps; ul < U; ul += kVWarps) {
+          for (int ul = (qd + 4 - u0 % 4) % 4; ul < U; ul += 4) {
             const int u = u0 + ul;
+            if (((u >> 2) & 1) != half) continue;                  // the other warp of this quadrant takes it
             const int ux = ul * 8;
             const int blk = u >> 2;
             const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
@@ -405,16 +409,6 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 const int ci = 3 * blk + dx, ds = ci % kDSlots;       // chunk index and its TMEM slot
                 if (!warp_wait(bar(kBarDFull + ds), (ci / kDSlots) & 1)) { ok = false; break; }
                 tc_fence_after_sync();
-                // one halo column of the strip, rows 0..5, widened to fp32 once
-                float vf[6][8];
-#pragma unroll
-                for (int r = 0; r < 6; ++r) {
-                    const uint4 v = lds_u4(sV, off0 + (uint32_t)(r * HW2 + dx) * 64u);
-                    vf[r][0] = bf16_lo(v.x); vf[r][1] = bf16_hi(v.x);
-                    vf[r][2] = bf16_lo(v.y); vf[r][3] = bf16_hi(v.y);
-                    vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
-                    vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
-                }
                 const uint32_t colbase = ds * kDSlotCols;
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
@@ -422,15 +416,24 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     float d[48];
                     const uint32_t ta = tq + ((uint32_t)(16 * mt) << 16) + colbase;
                     tmem_ld3_16x256b_x4(ta, ta + 32, ta + 64, d);
+                    // halo rows 2mt .. 2mt+3 of column dx, widened to fp32
+                    float vf[4][8];
 #pragma unroll
-                    for (int dy = 0; dy < 3; ++dy) {
-                        const int r = 2 * mt + dy;                 // halo rows r (half 0) and r+1 (half 1)
+                    for (int r = 0; r < 4; ++r) {
+                        const uint4 v = lds_u4(sV, off0 + (uint32_t)((2 * mt + r) * HW2 + dx) * 64u);
+                        vf[r][0] = bf16_lo(v.x); vf[r][1] = bf16_hi(v.x);
+                        vf[r][2] = bf16_lo(v.y); vf[r][3] = bf16_hi(v.y);
+                        vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
+                        vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
+                    }
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy) {               // halo rows dy (half 0) and dy+1 (half 1)
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             ffma2(o_acc[2 * mt][2 * j], o_acc[2 * mt][2 * j + 1], d[16 * dy + 4 * j], d[16 * dy + 4 * j + 1],
-                                  vf[r][2 * j], vf[r][2 * j + 1]);
+                                  vf[dy][2 * j], vf[dy][2 * j + 1]);
                             ffma2(o_acc[2 * mt + 1][2 * j], o_acc[2 * mt + 1][2 * j + 1], d[16 * dy + 4 * j + 2], d[16 * dy + 4 * j + 3],
-                                  vf[r + 1][2 * j], vf[r + 1][2 * j + 1]);
+                                  vf[dy + 1][2 * j], vf[dy + 1][2 * j + 1]);
                         }
                     }
                 }
@@ -467,7 +470,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
         }
         // quadrants of the last block that hold no unit: keep the chunk barriers in step
-        if (ok && my_blocks > 0 && (my_units & 3) != 0 && warp >= (my_units & 3)) {
+        if (ok && my_blocks > 0 && (my_units & 3) != 0 && qd >= (my_units & 3) && ((my_blocks - 1) & 1) == half) {
             for (int dx = 0; ok && dx < 3; ++dx) {
                 const int ci = 3 * (my_blocks - 1) + dx, ds = ci % kDSlots;
                 if (!warp_wait(bar(kBarDFull + ds), (ci / kDSlots) & 1)) { ok = false; break; }

@@ -18,15 +18,17 @@
 //                                                       D_v[c][8][t], [t == 8], [t == 8], 0 ...
 //   16 more columns hold 0 | 1 | 1 | 0,1,1,0... and so deliver sum_s e[p,s].
 // D (fp32) lives in tensor memory, pixel = TMEM lane.  Columns are ordered by tap column dx; the
-// three taps of one dx (96 columns; the last dx also carries the 16 sum columns) form a chunk, and
-// chunks go round a ring of four 112-column TMEM slots, so the MMA of a chunk is issued about one
-// block ahead of the value warps that read it.  Value warp w reads TMEM lanes 32w .. 32w+31 (its
+// three taps of one dx (96 columns; the last dx also carries the 16 sum columns) form a chunk.  The
+// two sets of value warps (even / odd blocks) each own two 112-column TMEM slots and walk them as
+// a ring, so while a set reads one chunk the MMA of its next chunk is already running.  Value warp w reads TMEM lanes 32w .. 32w+31 (its
 // quadrant) with tcgen05.ld.16x256b, whose register layout equals the mma.sync accumulator fragment.
 //
 // Roles (16 warps, 128 registers each): warps 0-7 value warps (warp % 4 = TMEM quadrant = unit index
 // within a block; warps w and w+4 take alternate blocks), warps 8-14 key warps (their B fragments
 // are re-read from shared memory for every unit), warp 15 allocates / frees tensor memory and its
-// lane 0 is the scheduler: it issues the TMA loads and the MMAs.  Every wait is bounded; a wait that runs out sets
+// lane 0 is the scheduler: it issues the TMA loads and the MMAs.  K (+ q) tiles and V tiles travel
+// in separate TMA rings, so the key warps can run ahead of the value warps by as many blocks as
+// there are A tiles.  Every wait is bounded; a wait that runs out sets
 // the status word, and tensor memory is released on every path.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -40,8 +42,9 @@ constexpr int kVWarps = 8;
 constexpr int kKWarps = 7;
 constexpr int kCtlWarp = kVWarps + kKWarps;             // warp 15
 constexpr int kThreads = (kVWarps + kKWarps + 1) * 32;
-constexpr int kMaxStages = 3;
-constexpr int kABufs = 2;                               // A tiles (one per block in flight)
+constexpr int kKStages = 2;                             // ring of K halo + q tiles
+constexpr int kMaxVStages = 4;                          // ring of V halo tiles
+constexpr int kABufs = 4;                               // A tiles (one per block in flight)
 constexpr int kBkBytes = 9 * 2 * 32 * 16;               // key-side B fragments of the head, fragment order
 constexpr int kABytes = 128 * 64;                       // 128 rows x 32 bf16
 constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
@@ -49,7 +52,7 @@ constexpr int kBBytes = kBCols * 64;
 constexpr int kWeightBytes = kHeadDim * 81 * 4;         // fp32 weights of one head, one side
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kTmemCols = 512;
-constexpr int kDSlots = 4;                              // ring of TMEM chunks
+constexpr int kDSlots = 4;                              // two TMEM chunk slots per value-warp set
 constexpr uint32_t kDSlotCols = 112;
 constexpr uint32_t kIdesc96 = umma_idesc_bf16(128, 96);
 constexpr uint32_t kIdesc112 = umma_idesc_bf16(128, 112);
@@ -63,13 +66,14 @@ struct UmmaParams {
     int B, H, W, heads;
     int TW;                    // tile width in pixels (multiple of 8); tile height is 4
     int tiles_x, tiles_y;
-    int stages;                // 2 or 3
+    int stages;                // depth of the V ring (2..4)
     float scale_log2e;         // log2(e) / sqrt(head_dim)
 };
 
 struct Smem {
     uint32_t halo_pad;         // bytes of one K or V halo tile (6 rows x (TW+2) pixels x 64 B), 1024-aligned
-    uint32_t stage_bytes;      // K halo | V halo | q tile
+    uint32_t kstage_bytes;     // K halo | q tile
+    uint32_t v_off;            // V ring [vstages][halo_pad]
     uint32_t b_off;            // B tile of the value-side MMA
     uint32_t bk_off;           // key-side B fragments [tap][k-step][lane][4 words]
     uint32_t a_off;            // A tiles [kABufs][kABytes]
@@ -78,14 +82,15 @@ struct Smem {
     uint32_t total;            // including 1024 bytes of slack to align the base
 };
 
-__host__ __device__ inline Smem smem_layout(int TW, int stages) {
+__host__ __device__ inline Smem smem_layout(int TW, int vstages) {
     Smem s;
     s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 1023u) & ~1023u;
-    s.stage_bytes = 2 * s.halo_pad + (((uint32_t)(4 * TW * 64) + 1023u) & ~1023u);
-    // the last stage doubles as the staging area of the head's fp32 weights (both sides)
+    // a V stage doubles as the staging area of the head's fp32 weights (both sides)
     const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
-    if (s.stage_bytes < wbytes) s.stage_bytes = wbytes;
-    s.b_off = s.stage_bytes * stages;
+    if (s.halo_pad < wbytes) s.halo_pad = wbytes;
+    s.kstage_bytes = s.halo_pad + (((uint32_t)(4 * TW * 64) + 1023u) & ~1023u);
+    s.v_off = kKStages * s.kstage_bytes;
+    s.b_off = s.v_off + vstages * s.halo_pad;
     s.bk_off = s.b_off + kBBytes;
     s.a_off = s.bk_off + kBkBytes;
     s.tmem_off = s.a_off + kABufs * kABytes;
@@ -95,15 +100,17 @@ __host__ __device__ inline Smem smem_layout(int TW, int stages) {
 }
 
 // barrier indices (8 bytes each) behind bar_off
-constexpr int kBarFull = 0;          // [stage]  TMA landed
-constexpr int kBarEmpty = 3;         // [stage]  every key and value warp is done with the stage
-constexpr int kBarWeights = 6;       // weights landed
-constexpr int kBarWeightsDone = 7;   // all warps have built their fragments / their share of the B tile
-constexpr int kBarAReady = 8;        // [A buffer]  the 4 units of a block have written their rows
-constexpr int kBarAFree = 11;        // [A buffer]  the MMAs reading the buffer are complete
-constexpr int kBarDFull = 14;        // [TMEM slot]  MMA results of a chunk are in tensor memory
-constexpr int kBarDFree = 18;        // [TMEM slot]  the 4 value warps are done reading the chunk
-constexpr int kBarVDone = 22;        // value warps have finished all TMEM reads
+constexpr int kBarKFull = 0;         // [K stage]  K halo and q tile landed
+constexpr int kBarKEmpty = 2;        // [K stage]  every key warp is done with the stage
+constexpr int kBarVFull = 4;         // [V stage]  V halo landed
+constexpr int kBarVEmpty = 8;        // [V stage]  every value warp is done with the stage
+constexpr int kBarWeights = 12;      // weights landed
+constexpr int kBarWeightsDone = 13;  // all warps are done with the weight staging area
+constexpr int kBarAReady = 14;       // [A buffer]  the 4 units of a block have written their rows
+constexpr int kBarAFree = 18;        // [A buffer]  the MMAs reading the buffer are complete
+constexpr int kBarDFull = 22;        // [TMEM slot]  MMA results of a chunk are in tensor memory
+constexpr int kBarDFree = 26;        // [TMEM slot]  the 4 value warps of the set are done reading the chunk
+constexpr int kBarVDone = 30;        // value warps have finished all TMEM reads
 
 __device__ __forceinline__ float4 lds_f4(const unsigned char* base, uint32_t off) {
     return *reinterpret_cast<const float4*>(base + off);
@@ -129,7 +136,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tig = lane & 3;
-    const int S = P.stages;
+    const int SV = P.stages;                                   // V ring depth
     const int U = P.TW >> 3;                                   // units per tile
     const int HW2 = P.TW + 2;
 
@@ -144,9 +151,13 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     const int C = P.heads * kHeadDim;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxStages; ++s) {
-            mbar_init(bar(kBarFull + s), 1);
-            mbar_init(bar(kBarEmpty + s), kKWarps + kVWarps);
+        for (int s = 0; s < kKStages; ++s) {
+            mbar_init(bar(kBarKFull + s), 1);
+            mbar_init(bar(kBarKEmpty + s), kKWarps);
+        }
+        for (int s = 0; s < kMaxVStages; ++s) {
+            mbar_init(bar(kBarVFull + s), 1);
+            mbar_init(bar(kBarVEmpty + s), kVWarps);
         }
         mbar_init(bar(kBarWeights), 1);
         mbar_init(bar(kBarWeightsDone), kKWarps + kVWarps + 1);
@@ -169,30 +180,42 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     tc_fence_after_sync();
     const uint32_t tmem = *reinterpret_cast<const volatile uint32_t*>(smem + L.tmem_off);
 
-    // tile n of this CTA -> stage n % S
-    auto issue_tile = [&](int n) {
+    // tile n of this CTA -> K stage n % kKStages, V stage n % SV
+    auto tile_coords = [&](int n, int& tx, int& ty, int& b) {
         const int gt = rank + n * nrank;
-        const int tx = gt % P.tiles_x;
-        const int ty = (gt / P.tiles_x) % P.tiles_y;
-        const int b = gt / (P.tiles_x * P.tiles_y);
-        const int s = n % S;
-        const uint32_t base = smem_u32(smem + (size_t)s * L.stage_bytes);
-        const uint32_t fb = bar(kBarFull + s);
-        mbar_expect_tx(fb, (uint32_t)(2 * 6 * HW2 * 64 + 4 * P.TW * 64));
+        tx = gt % P.tiles_x;
+        ty = (gt / P.tiles_x) % P.tiles_y;
+        b = gt / (P.tiles_x * P.tiles_y);
+    };
+    auto issue_k_tile = [&](int n) {
+        int tx, ty, b;
+        tile_coords(n, tx, ty, b);
+        const int s = n % kKStages;
+        const uint32_t base = smem_u32(smem + (size_t)s * L.kstage_bytes);
+        const uint32_t fb = bar(kBarKFull + s);
+        mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64 + 4 * P.TW * 64));
         tma_load_4d(base, &map_k, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
-        tma_load_4d(base + L.halo_pad, &map_v, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
-        tma_load_4d(base + 2 * L.halo_pad, &map_q, fb, h * kHeadDim, tx * P.TW, ty * 4, b);
+        tma_load_4d(base + L.halo_pad, &map_q, fb, h * kHeadDim, tx * P.TW, ty * 4, b);
+    };
+    auto issue_v_tile = [&](int n) {
+        int tx, ty, b;
+        tile_coords(n, tx, ty, b);
+        const int s = n % SV;
+        const uint32_t fb = bar(kBarVFull + s);
+        mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64));
+        tma_load_4d(smem_u32(smem + L.v_off + (size_t)s * L.halo_pad), &map_v, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
     };
 
-    // The fp32 weights of the head are staged in the LAST stage's memory; that stage receives its
+    // The fp32 weights of the head are staged in the LAST V stage's memory; that stage receives its
     // first tile only after every warp has finished with them.
-    const unsigned char* w_stage = smem + (size_t)(S - 1) * L.stage_bytes;
-    int issued = 0;                                            // producer state (control warp, lane 0)
+    const unsigned char* w_stage = smem + L.v_off + (size_t)(SV - 1) * L.halo_pad;
+    int k_issued = 0, v_issued = 0;                            // scheduler state (control warp, lane 0)
     if (my_tiles > 0 && warp == kCtlWarp && lane == 0) {
         mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
         bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
         bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
-        while (issued < my_tiles && issued < S - 1) issue_tile(issued++);
+        while (k_issued < my_tiles && k_issued < kKStages) issue_k_tile(k_issued++);
+        while (v_issued < my_tiles && v_issued < SV - 1) issue_v_tile(v_issued++);
     }
     __syncwarp();
 
@@ -273,14 +296,14 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         // a tile in which it owns no unit: a warp that skipped a phase of a barrier could later
         // mistake an older phase for the one it waits for.
         for (int ti = 0; ok && ti < my_tiles; ++ti) {
-            const int stage = ti % S;
-            if (!warp_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
+            const int stage = ti % kKStages;
+            if (!warp_wait(bar(kBarKFull + stage), (ti / kKStages) & 1)) { ok = false; break; }
             const int u0 = ti * U;
           for (int ul = (kw + kKWarps - u0 % kKWarps) % kKWarps; ul < U; ul += kKWarps) {
             const int u = u0 + ul;
             const int ux = ul * 8;
-            const unsigned char* sK = smem + (size_t)stage * L.stage_bytes;
-            const unsigned char* sQ = sK + 2 * L.halo_pad;
+            const unsigned char* sK = smem + (size_t)stage * L.kstage_bytes;
+            const unsigned char* sQ = sK + L.halo_pad;
             // q of the lane's four pixels (rows 0..3 of column ux + g)
             uint32_t qf[4][4];
 #pragma unroll
@@ -370,7 +393,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             if (lane == 0) mbar_arrive(bar(kBarAReady + ab));
           }
             __syncwarp();
-            if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
+            if (ok && lane == 0) mbar_arrive(bar(kBarKEmpty + stage)); // this warp is done with the stage
         }
     } else if (warp < kVWarps) {
         // =====================================================================================
@@ -386,15 +409,15 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             const int tx = gt % P.tiles_x;
             const int ty = (gt / P.tiles_x) % P.tiles_y;
             const int b = gt / (P.tiles_x * P.tiles_y);
-            const int stage = ti % S;
-            if (!warp_wait(bar(kBarFull + stage), (ti / S) & 1)) { ok = false; break; }
+            const int stage = ti % SV;
+            if (!warp_wait(bar(kBarVFull + stage), (ti / SV) & 1)) { ok = false; break; }
             const int u0 = ti * U;
           for (int ul = (qd + 4 - u0 % 4) % 4; ul < U; ul += 4) {
             const int u = u0 + ul;
             if (((u >> 2) & 1) != half) continue;                  // the other warp of this quadrant takes it
             const int ux = ul * 8;
             const int blk = u >> 2;
-            const unsigned char* sV = smem + (size_t)stage * L.stage_bytes + L.halo_pad;
+            const unsigned char* sV = smem + L.v_off + (size_t)stage * L.halo_pad;
             const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
 
             float o_acc[4][8];
@@ -406,8 +429,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
 
 #pragma unroll
             for (int dx = 0; dx < 3; ++dx) {
-                const int ci = 3 * blk + dx, ds = ci % kDSlots;       // chunk index and its TMEM slot
-                if (!warp_wait(bar(kBarDFull + ds), (ci / kDSlots) & 1)) { ok = false; break; }
+                const int cs = 3 * (blk >> 1) + dx, ds = 2 * half + (cs & 1);   // chunk index within the set, TMEM slot
+                if (!warp_wait(bar(kBarDFull + ds), (cs >> 1) & 1)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t colbase = ds * kDSlotCols;
 #pragma unroll
@@ -467,13 +490,13 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             }
           }
             __syncwarp();
-            if (ok && lane == 0) mbar_arrive(bar(kBarEmpty + stage));  // this warp is done with the stage
+            if (ok && lane == 0) mbar_arrive(bar(kBarVEmpty + stage)); // this warp is done with the stage
         }
         // quadrants of the last block that hold no unit: keep the chunk barriers in step
         if (ok && my_blocks > 0 && (my_units & 3) != 0 && qd >= (my_units & 3) && ((my_blocks - 1) & 1) == half) {
             for (int dx = 0; ok && dx < 3; ++dx) {
-                const int ci = 3 * (my_blocks - 1) + dx, ds = ci % kDSlots;
-                if (!warp_wait(bar(kBarDFull + ds), (ci / kDSlots) & 1)) { ok = false; break; }
+                const int cs = 3 * ((my_blocks - 1) >> 1) + dx, ds = 2 * half + (cs & 1);
+                if (!warp_wait(bar(kBarDFull + ds), (cs >> 1) & 1)) { ok = false; break; }
                 if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
             }
         }
@@ -493,30 +516,43 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             //   its TMEM slot has been read.
             // It gives up when nothing has moved for about two seconds.
             const uint32_t sA0 = smem_u32(smem + L.a_off), sB0 = smem_u32(smem + L.b_off);
-            bool weights_done = false, a_ready = false;
-            int blk = 0, dx = 0;
+            bool weights_done = false;
+            int qblk[2] = {0, 1}, qdx[2] = {0, 0};                  // MMA queue of each value-warp set
+            bool stood_in = false;
             long long last_progress = clock64();
-            while (issued < my_tiles || blk < my_blocks) {
+            while (k_issued < my_tiles || v_issued < my_tiles || qblk[0] < my_blocks || qblk[1] < my_blocks) {
                 bool progress = false;
                 if (!weights_done && mbar_test(bar(kBarWeightsDone), 0)) { weights_done = true; progress = true; }
-                if (issued < my_tiles) {
-                    bool free_now;
-                    if (issued < S - 1) free_now = true;
-                    else if (issued == S - 1) free_now = weights_done;          // staging area must be dead
-                    else free_now = mbar_test(bar(kBarEmpty + issued % S), ((issued / S) - 1) & 1);
-                    if (free_now) { issue_tile(issued++); progress = true; }
+                if (k_issued < my_tiles &&
+                    (k_issued < kKStages || mbar_test(bar(kBarKEmpty + k_issued % kKStages), ((k_issued / kKStages) - 1) & 1))) {
+                    issue_k_tile(k_issued++);
+                    progress = true;
                 }
-                if (blk < my_blocks && weights_done) {
-                    const int ab = blk % kABufs;
-                    if (dx == 0 && !a_ready) {
-                        if (blk == my_blocks - 1 && (my_units & 3) != 0) {       // partial last block: stand in
-                            for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
-                        }
-                        a_ready = true;                                          // now only the barrier decides
+                if (v_issued < my_tiles) {
+                    bool free_now;
+                    if (v_issued < SV - 1) free_now = true;
+                    else if (v_issued == SV - 1) free_now = weights_done;       // staging area must be dead
+                    else free_now = mbar_test(bar(kBarVEmpty + v_issued % SV), ((v_issued / SV) - 1) & 1);
+                    if (free_now) { issue_v_tile(v_issued++); progress = true; }
+                }
+                if (weights_done && !stood_in && my_blocks > 0 && (my_units & 3) != 0) {
+                    // partial last block: stand in for the units that do not exist.  No key warp can be
+                    // writing that A buffer for an earlier block any more once its AFree phase is over.
+                    const int lb = my_blocks - 1, ab = lb % kABufs;
+                    if (mbar_test(bar(kBarAFree + ab), ((lb / kABufs) & 1) ^ 1)) {
+                        for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
+                        stood_in = true;
+                        progress = true;
                     }
-                    const int ci = 3 * blk + dx, ds = ci % kDSlots;
+                }
+#pragma unroll
+                for (int set = 0; set < 2; ++set) {
+                    const int blk = qblk[set], dx = qdx[set];
+                    if (!weights_done || blk >= my_blocks) continue;
+                    const int ab = blk % kABufs;
+                    const int cs = 3 * (blk >> 1) + dx, ds = 2 * set + (cs & 1);
                     if (mbar_test(bar(kBarAReady + ab), (blk / kABufs) & 1) &&
-                        mbar_test(bar(kBarDFree + ds), ((ci / kDSlots) & 1) ^ 1)) {
+                        mbar_test(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1)) {
                         tc_fence_after_sync();
                         // columns dx*96 .. of B; K = 32 = two instructions of K = 16 (256 bytes apart)
                         const uint32_t sA = sA0 + ab * kABytes, sB = sB0 + dx * 12 * 512;
@@ -525,7 +561,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                         umma_bf16_ss(dcol, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB, 128, 512), idesc, 0);
                         umma_bf16_ss(dcol, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB + 256, 128, 512), idesc, 1);
                         umma_commit(bar(kBarDFull + ds));
-                        if (++dx == 3) { umma_commit(bar(kBarAFree + ab)); dx = 0; ++blk; a_ready = false; }
+                        if (dx == 2) { umma_commit(bar(kBarAFree + ab)); qdx[set] = 0; qblk[set] = blk + 2; }
+                        else qdx[set] = dx + 1;
                         progress = true;
                     }
                 }
@@ -605,7 +642,9 @@ cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream
     P.TW = TW;
     P.tiles_x = (p.W + TW - 1) / TW;
     P.tiles_y = (p.H + 3) / 4;
-    P.stages = smem_layout(TW, 3).total <= kMaxSmem ? 3 : 2;
+    P.stages = 2;                                          // V ring depth: as deep as fits
+    for (int st = kMaxVStages; st >= 2; --st)
+        if (smem_layout(TW, st).total <= kMaxSmem) { P.stages = st; break; }
     P.scale_log2e = kLog2e / sqrtf((float)kHeadDim);
     const Smem L = smem_layout(TW, P.stages);
     if (L.total > kMaxSmem) return cudaErrorInvalidConfiguration;

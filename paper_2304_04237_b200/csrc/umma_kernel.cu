@@ -535,21 +535,17 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     else free_now = mbar_test(bar(kBarVEmpty + v_issued % SV), ((v_issued / SV) - 1) & 1);
                     if (free_now) { issue_v_tile(v_issued++); progress = true; }
                 }
-                if (weights_done && !stood_in && my_blocks > 0 && (my_units & 3) != 0) {
-                    // partial last block: stand in for the units that do not exist.  No key warp can be
-                    // writing that A buffer for an earlier block any more once its AFree phase is over.
-                    const int lb = my_blocks - 1, ab = lb % kABufs;
-                    if (mbar_test(bar(kBarAFree + ab), ((lb / kABufs) & 1) ^ 1)) {
-                        for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
-                        stood_in = true;
-                        progress = true;
-                    }
-                }
 #pragma unroll
                 for (int set = 0; set < 2; ++set) {
                     const int blk = qblk[set], dx = qdx[set];
                     if (!weights_done || blk >= my_blocks) continue;
                     const int ab = blk % kABufs;
+                    if (!stood_in && blk == my_blocks - 1 && (my_units & 3) != 0) {
+                        // partial last block: stand in for the units that do not exist.  The queue has
+                        // reached this block, so the previous phase of its AReady barrier is over.
+                        for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
+                        stood_in = true;
+                    }
                     const int cs = 3 * (blk >> 1) + dx, ds = 2 * set + (cs & 1);
                     if (mbar_test(bar(kBarAReady + ab), (blk / kABufs) & 1) &&
                         mbar_test(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1)) {
@@ -570,7 +566,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     last_progress = clock64();
                 } else {
                     if (clock64() - last_progress > 4000000000LL) { ok = false; break; }
-                    __nanosleep(40);
+                    __nanosleep(100);
                 }
             }
         }

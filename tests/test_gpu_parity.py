@@ -198,6 +198,43 @@ def test_deterministic_and_leaves_guard_bands_alone(variant):
         sa.slide_attn_destroy(ctx)
 
 
+@pytest.mark.parametrize("variant", ["mma_ws", "umma"])
+def test_pipelined_variants_many_shapes_repeatable(variant):
+    """The persistent kernels hand work between warps through mbarrier rings; shapes with many or
+    few tiles per CTA, partial last blocks and ragged widths must all give the DIRECT variant's
+    result (within the bf16 tolerance of both) and the same bits on every repetition."""
+    shapes = [(64, 56, 56, 3), (7, 56, 56, 2), (33, 28, 28, 6), (5, 28, 42, 6), (2, 128, 128, 3),
+              (1, 4, 8, 1), (9, 12, 72, 1), (130, 8, 8, 2), (3, 61, 67, 5)]
+    for (B, H, W, heads) in shapes:
+        g = torch.Generator(device="cuda").manual_seed(B * 1000 + W)
+        q = torch.randn(B, H, W, heads, 32, device="cuda", generator=g).bfloat16()
+        k = torch.randn(B, H, W, heads, 32, device="cuda", generator=g).bfloat16()
+        v = torch.randn(B, H, W, heads, 32, device="cuda", generator=g).bfloat16()
+        C = heads * 32
+        wk = torch.eye(9, device="cuda").repeat(C, 1, 1).contiguous() + 0.05 * torch.randn(C, 9, 9, device="cuda", generator=g)
+        wv = torch.eye(9, device="cuda").repeat(C, 1, 1).contiguous() + 0.05 * torch.randn(C, 9, 9, device="cuda", generator=g)
+        bias = 0.1 * torch.randn(heads, 9, device="cuda", generator=g)
+        ctx = sa.slide_attn_create(B, H, W, heads, 32, 3, torch.bfloat16, True)
+        try:
+            ref = torch.empty_like(q)
+            sa.slide_attn_set_variant(ctx, sa.VARIANT_DIRECT)
+            sa.slide_attn_forward(ctx, q, k, v, wk, wv, bias, ref)
+            sa.slide_attn_set_variant(ctx, VARIANTS[variant])
+            outs = []
+            for _ in range(4):
+                o = torch.full_like(q, float("nan"))
+                sa.slide_attn_forward(ctx, q, k, v, wk, wv, bias, o)
+                outs.append(o)
+            torch.cuda.synchronize()
+            assert sa.slide_attn_query_status(ctx) == sa.OK, (variant, B, H, W, heads)
+            for o in outs[1:]:
+                assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16)), (variant, B, H, W, heads)
+            err = (outs[0].float() - ref.float()).abs() / ref.float().abs().clamp(min=1.0)
+            assert float(err.max()) <= 2.5e-2, (variant, B, H, W, heads, float(err.max()))
+        finally:
+            sa.slide_attn_destroy(ctx)
+
+
 def test_forward_argument_errors():
     x = synth.make_inputs(1, 4, 4, 1, 32, 3, "f32", seed=1, has_bias=True)
     dev = to_device(x, "f32")

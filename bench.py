@@ -44,6 +44,28 @@ def algorithmic_bytes(cfg) -> int:
     return n * C * 4 * sz + 2 * C * k2 * k2 * 4 + (cfg["heads"] * k2 * 4 if cfg["has_bias"] else 0)
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant kernel
+# from one `ncu --set full` capture (profiles/).  It is tied to the kernel source by a hash: once
+# the kernel changes, the figure no longer applies and `traffic` is reported as null.
+NCU_TRAFFIC = {
+    ("umma", "c2"): {"bytes": 82.18e6,
+                     "sources": ("paper_2304_04237_b200/csrc/umma_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
+                     "sha256": "8ee66de4813a0a664e8d280a610dace4e6544e630ad8c6f2f771a5c5ad1011c4"},
+}
+
+
+def ncu_traffic(variant, workload):
+    import hashlib
+    rec = NCU_TRAFFIC.get((variant, workload))
+    if rec is None:
+        return None
+    try:
+        h = hashlib.sha256(b"".join(open(os.path.join(ROOT, f), "rb").read() for f in rec["sources"])).hexdigest()
+    except OSError:
+        return None
+    return rec["bytes"] if h == rec["sha256"] else None
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -319,7 +341,8 @@ def main():
             "variant": variant, "gpu_launches": launches * args.steps,
             "hbm_gbs_algorithmic": abytes / (ms_per_step * 1e-3) / 1e9,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": (achieved / peak if achieved else None), "traffic": None,
+                         "frac": (achieved / peak if achieved else None),
+                         "traffic": ncu_traffic(variant, args.workload),
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": abytes,
                          "kernel_ms": main_ms, "forward_ms": fwd_ms, "launches_averaged": n_prof},
             "clocks": clocks, "e2e": e2e,

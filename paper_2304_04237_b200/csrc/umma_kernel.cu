@@ -180,42 +180,53 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     tc_fence_after_sync();
     const uint32_t tmem = *reinterpret_cast<const volatile uint32_t*>(smem + L.tmem_off);
 
-    // tile n of this CTA -> K stage n % kKStages, V stage n % SV
-    auto tile_coords = [&](int n, int& tx, int& ty, int& b) {
-        const int gt = rank + n * nrank;
-        tx = gt % P.tiles_x;
-        ty = (gt / P.tiles_x) % P.tiles_y;
-        b = gt / (P.tiles_x * P.tiles_y);
+    // Tile n of this CTA is global tile rank + n * nrank -> K stage n % kKStages, V stage n % SV.
+    // Whoever walks the tiles keeps (tx, ty, b) and a stage counter and steps them without dividing:
+    // a division costs a lone thread some hundred cycles, and the control thread has none to spare.
+    struct TileWalk { int tx, ty, b, stage, round; };
+    const int step_tx = nrank % P.tiles_x, step_ty = (nrank / P.tiles_x) % P.tiles_y,
+              step_b = nrank / (P.tiles_x * P.tiles_y);
+    auto walk_begin = [&]() {
+        TileWalk w;
+        w.tx = rank % P.tiles_x;
+        w.ty = (rank / P.tiles_x) % P.tiles_y;
+        w.b = rank / (P.tiles_x * P.tiles_y);
+        w.stage = 0; w.round = 0;
+        return w;
     };
-    auto issue_k_tile = [&](int n) {
-        int tx, ty, b;
-        tile_coords(n, tx, ty, b);
-        const int s = n % kKStages;
-        const uint32_t base = smem_u32(smem + (size_t)s * L.kstage_bytes);
-        const uint32_t fb = bar(kBarKFull + s);
+    auto walk_next = [&](TileWalk& w, int nstages) {
+        w.tx += step_tx;
+        if (w.tx >= P.tiles_x) { w.tx -= P.tiles_x; ++w.ty; }
+        w.ty += step_ty;
+        if (w.ty >= P.tiles_y) { w.ty -= P.tiles_y; ++w.b; }
+        w.b += step_b;
+        if (++w.stage == nstages) { w.stage = 0; ++w.round; }
+    };
+    auto issue_k_tile = [&](const TileWalk& w) {
+        const uint32_t base = smem_u32(smem + (size_t)w.stage * L.kstage_bytes);
+        const uint32_t fb = bar(kBarKFull + w.stage);
         mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64 + 4 * P.TW * 64));
-        tma_load_4d(base, &map_k, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
-        tma_load_4d(base + L.halo_pad, &map_q, fb, h * kHeadDim, tx * P.TW, ty * 4, b);
+        tma_load_4d(base, &map_k, fb, h * kHeadDim, w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
+        tma_load_4d(base + L.halo_pad, &map_q, fb, h * kHeadDim, w.tx * P.TW, w.ty * 4, w.b);
     };
-    auto issue_v_tile = [&](int n) {
-        int tx, ty, b;
-        tile_coords(n, tx, ty, b);
-        const int s = n % SV;
-        const uint32_t fb = bar(kBarVFull + s);
+    auto issue_v_tile = [&](const TileWalk& w) {
+        const uint32_t fb = bar(kBarVFull + w.stage);
         mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64));
-        tma_load_4d(smem_u32(smem + L.v_off + (size_t)s * L.halo_pad), &map_v, fb, h * kHeadDim, tx * P.TW - 1, ty * 4 - 1, b);
+        tma_load_4d(smem_u32(smem + L.v_off + (size_t)w.stage * L.halo_pad), &map_v, fb, h * kHeadDim,
+                    w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
     };
 
     // The fp32 weights of the head are staged in the LAST V stage's memory; that stage receives its
     // first tile only after every warp has finished with them.
     const unsigned char* w_stage = smem + L.v_off + (size_t)(SV - 1) * L.halo_pad;
     int k_issued = 0, v_issued = 0;                            // scheduler state (control warp, lane 0)
+    TileWalk kq = walk_begin(), vq = kq;                       // next tile of the K queue / of the V queue
     if (my_tiles > 0 && warp == kCtlWarp && lane == 0) {
         mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
         bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
         bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
-        while (k_issued < my_tiles && k_issued < kKStages) issue_k_tile(k_issued++);
-        while (v_issued < my_tiles && v_issued < SV - 1) issue_v_tile(v_issued++);
+        while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
+        while (v_issued < my_tiles && v_issued < SV - 1) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
     }
     __syncwarp();
 
@@ -404,13 +415,10 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         const int qd = warp & 3, half = warp >> 2;                 // quadrant; which blocks (even / odd)
         const uint32_t tq = tmem + ((uint32_t)(32 * qd) << 16);
 
-        for (int ti = 0; ok && ti < my_tiles; ++ti) {
-            const int gt = rank + ti * nrank;
-            const int tx = gt % P.tiles_x;
-            const int ty = (gt / P.tiles_x) % P.tiles_y;
-            const int b = gt / (P.tiles_x * P.tiles_y);
-            const int stage = ti % SV;
-            if (!warp_wait(bar(kBarVFull + stage), (ti / SV) & 1)) { ok = false; break; }
+        TileWalk vw = walk_begin();
+        for (int ti = 0; ok && ti < my_tiles; ++ti, walk_next(vw, SV)) {
+            const int tx = vw.tx, ty = vw.ty, b = vw.b, stage = vw.stage;
+            if (!warp_wait(bar(kBarVFull + stage), vw.round & 1)) { ok = false; break; }
             const int u0 = ti * U;
           for (int ul = (qd + 4 - u0 % 4) % 4; ul < U; ul += 4) {
             const int u = u0 + ul;
@@ -524,16 +532,16 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 bool progress = false;
                 if (!weights_done && mbar_test(bar(kBarWeightsDone), 0)) { weights_done = true; progress = true; }
                 if (k_issued < my_tiles &&
-                    (k_issued < kKStages || mbar_test(bar(kBarKEmpty + k_issued % kKStages), ((k_issued / kKStages) - 1) & 1))) {
-                    issue_k_tile(k_issued++);
+                    (kq.round == 0 || mbar_test(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1))) {
+                    issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued;
                     progress = true;
                 }
                 if (v_issued < my_tiles) {
                     bool free_now;
                     if (v_issued < SV - 1) free_now = true;
                     else if (v_issued == SV - 1) free_now = weights_done;       // staging area must be dead
-                    else free_now = mbar_test(bar(kBarVEmpty + v_issued % SV), ((v_issued / SV) - 1) & 1);
-                    if (free_now) { issue_v_tile(v_issued++); progress = true; }
+                    else free_now = mbar_test(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
+                    if (free_now) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; progress = true; }
                 }
 #pragma unroll
                 for (int set = 0; set < 2; ++set) {

@@ -111,6 +111,16 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 
 // One non-blocking probe of a phase.
+// Same test as a 0/1 word, without a branch: several can be in flight before the first is used.
+__device__ __forceinline__ uint32_t mbar_test_u32(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done;
+}
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     uint32_t done;
     asm volatile(

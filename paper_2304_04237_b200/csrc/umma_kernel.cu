@@ -524,58 +524,57 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             //   its TMEM slot has been read.
             // It gives up when nothing has moved for about two seconds.
             const uint32_t sA0 = smem_u32(smem + L.a_off), sB0 = smem_u32(smem + L.b_off);
+            // Every pass first puts all its barrier tests in flight together and only then acts on
+            // them: this thread shares its scheduler with three busy warps, and tests taken one
+            // after the other, each behind a branch, made a pass cost as much as a whole chunk.
             bool weights_done = false;
-            int qblk[2] = {0, 1}, qdx[2] = {0, 0};                  // MMA queue of each value-warp set
+            int blk0 = 0, blk1 = 1, dx0 = 0, dx1 = 0;                // MMA queue of each value-warp set
             bool stood_in = false;
-            long long last_progress = clock64();
-            while (k_issued < my_tiles || v_issued < my_tiles || qblk[0] < my_blocks || qblk[1] < my_blocks) {
-                bool progress = false;
-                if (!weights_done && mbar_test(bar(kBarWeightsDone), 0)) { weights_done = true; progress = true; }
-                if (k_issued < my_tiles &&
-                    (kq.round == 0 || mbar_test(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1))) {
-                    issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued;
-                    progress = true;
+            const int partial = (my_units & 3) != 0 ? my_blocks - 1 : -1;   // block with fewer than 4 units
+            int left = 2 * my_tiles - k_issued - v_issued + 3 * my_blocks;  // actions still to issue
+            uint32_t idle = 0;
+            auto issue_chunk = [&](int set, int& blk, int& dx) {
+                const int ab = blk % kABufs, cs = 3 * (blk >> 1) + dx, ds = 2 * set + (cs & 1);
+                tc_fence_after_sync();
+                // columns dx*96 .. of B; K = 32 = two instructions of K = 16 (256 bytes apart)
+                const uint32_t sA = sA0 + ab * kABytes, sB = sB0 + dx * 12 * 512;
+                const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
+                const uint32_t dcol = tmem + ds * kDSlotCols;
+                umma_bf16_ss(dcol, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB, 128, 512), idesc, 0);
+                umma_bf16_ss(dcol, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB + 256, 128, 512), idesc, 1);
+                umma_commit(bar(kBarDFull + ds));
+                if (dx == 2) { umma_commit(bar(kBarAFree + ab)); dx = 0; blk += 2; }
+                else ++dx;
+                --left;
+            };
+            while (left > 0) {
+                if (!weights_done) weights_done = mbar_test(bar(kBarWeightsDone), 0);
+                if (!stood_in && (blk0 == partial || blk1 == partial)) {
+                    // partial last block: stand in for the units that do not exist.  A queue has
+                    // reached this block, so the previous phase of its AReady barrier is over.
+                    for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + partial % kABufs));
+                    stood_in = true;
                 }
-                if (v_issued < my_tiles) {
-                    bool free_now;
-                    if (v_issued < SV - 1) free_now = true;
-                    else if (v_issued == SV - 1) free_now = weights_done;       // staging area must be dead
-                    else free_now = mbar_test(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
-                    if (free_now) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; progress = true; }
+                // A stage or slot in its first round is free: parity 1 of a fresh barrier tests true.
+                const int cs0 = 3 * (blk0 >> 1) + dx0, cs1 = 3 * (blk1 >> 1) + dx1;
+                const uint32_t tK = mbar_test_u32(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1);
+                const uint32_t tV = mbar_test_u32(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
+                const uint32_t tA0 = mbar_test_u32(bar(kBarAReady + blk0 % kABufs), (blk0 / kABufs) & 1);
+                const uint32_t tD0 = mbar_test_u32(bar(kBarDFree + (cs0 & 1)), ((cs0 >> 1) & 1) ^ 1);
+                const uint32_t tA1 = mbar_test_u32(bar(kBarAReady + blk1 % kABufs), (blk1 / kABufs) & 1);
+                const uint32_t tD1 = mbar_test_u32(bar(kBarDFree + 2 + (cs1 & 1)), ((cs1 >> 1) & 1) ^ 1);
+                const int left_before = left;
+                if (tK != 0 && k_issued < my_tiles) {
+                    issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; --left;
                 }
-#pragma unroll
-                for (int set = 0; set < 2; ++set) {
-                    const int blk = qblk[set], dx = qdx[set];
-                    if (!weights_done || blk >= my_blocks) continue;
-                    const int ab = blk % kABufs;
-                    if (!stood_in && blk == my_blocks - 1 && (my_units & 3) != 0) {
-                        // partial last block: stand in for the units that do not exist.  The queue has
-                        // reached this block, so the previous phase of its AReady barrier is over.
-                        for (int m = my_units & 3; m < 4; ++m) mbar_arrive(bar(kBarAReady + ab));
-                        stood_in = true;
-                    }
-                    const int cs = 3 * (blk >> 1) + dx, ds = 2 * set + (cs & 1);
-                    if (mbar_test(bar(kBarAReady + ab), (blk / kABufs) & 1) &&
-                        mbar_test(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1)) {
-                        tc_fence_after_sync();
-                        // columns dx*96 .. of B; K = 32 = two instructions of K = 16 (256 bytes apart)
-                        const uint32_t sA = sA0 + ab * kABytes, sB = sB0 + dx * 12 * 512;
-                        const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
-                        const uint32_t dcol = tmem + ds * kDSlotCols;
-                        umma_bf16_ss(dcol, umma_smem_desc(sA, 128, 512), umma_smem_desc(sB, 128, 512), idesc, 0);
-                        umma_bf16_ss(dcol, umma_smem_desc(sA + 256, 128, 512), umma_smem_desc(sB + 256, 128, 512), idesc, 1);
-                        umma_commit(bar(kBarDFull + ds));
-                        if (dx == 2) { umma_commit(bar(kBarAFree + ab)); qdx[set] = 0; qblk[set] = blk + 2; }
-                        else qdx[set] = dx + 1;
-                        progress = true;
-                    }
+                // the last V stage held the weights: its first tile waits until every warp is done with them
+                if (tV != 0 && v_issued < my_tiles && (v_issued != SV - 1 || weights_done)) {
+                    issue_v_tile(vq); walk_next(vq, SV); ++v_issued; --left;
                 }
-                if (progress) {
-                    last_progress = clock64();
-                } else {
-                    if (clock64() - last_progress > 4000000000LL) { ok = false; break; }
-                    __nanosleep(100);
-                }
+                if ((tA0 & tD0) != 0 && blk0 < my_blocks) issue_chunk(0, blk0, dx0);
+                if ((tA1 & tD1) != 0 && blk1 < my_blocks) issue_chunk(1, blk1, dx1);
+                if (left != left_before) idle = 0;
+                else if (++idle > (1u << 24)) { ok = false; break; }      // nothing moved for seconds: give up
             }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;

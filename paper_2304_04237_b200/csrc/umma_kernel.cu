@@ -444,19 +444,26 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
                     // A'[pixel rows 2mt, 2mt+1][taps (dy = 0..2, dx)][8 channels]: three loads in flight
-                    float d[48];
+                    // while the halo rows 2mt .. 2mt+3 of column dx come out of shared memory
+                    uint32_t dr[48];
                     const uint32_t ta = tq + ((uint32_t)(16 * mt) << 16) + colbase;
-                    tmem_ld3_16x256b_x4(ta, ta + 32, ta + 64, d);
-                    // halo rows 2mt .. 2mt+3 of column dx, widened to fp32
-                    float vf[4][8];
+                    tmem_ld3_16x256b_x4_nowait(ta, ta + 32, ta + 64, dr);
+                    uint4 vp[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) vp[r] = lds_u4(sV, off0 + (uint32_t)((2 * mt + r) * HW2 + dx) * 64u);
+                    float vf[4][8];                                // widened to fp32
 #pragma unroll
                     for (int r = 0; r < 4; ++r) {
-                        const uint4 v = lds_u4(sV, off0 + (uint32_t)((2 * mt + r) * HW2 + dx) * 64u);
+                        const uint4 v = vp[r];
                         vf[r][0] = bf16_lo(v.x); vf[r][1] = bf16_hi(v.x);
                         vf[r][2] = bf16_lo(v.y); vf[r][3] = bf16_hi(v.y);
                         vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
                         vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
                     }
+                    tmem_wait_ld48(dr);
+                    float d[48];
+#pragma unroll
+                    for (int i = 0; i < 48; ++i) d[i] = __uint_as_float(dr[i]);
 #pragma unroll
                     for (int dy = 0; dy < 3; ++dy) {               // halo rows dy (half 0) and dy+1 (half 1)
 #pragma unroll
@@ -472,7 +479,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     float s0[4], s1[4];
                     tmem_ld_16x256b_x1(tq + colbase + 96, s0);                      // pixel rows 0, 1
                     tmem_ld_16x256b_x1(tq + (16u << 16) + colbase + 96, s1);        // pixel rows 2, 3
-                    inv[0] = 1.f / s0[0]; inv[1] = 1.f / s0[2]; inv[2] = 1.f / s1[0]; inv[3] = 1.f / s1[2];
+                    inv[0] = rcp_approx(s0[0]); inv[1] = rcp_approx(s0[2]); inv[2] = rcp_approx(s1[0]); inv[3] = rcp_approx(s1[2]);
                 }
                 tc_fence_before_sync();
                 __syncwarp();

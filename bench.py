@@ -50,7 +50,7 @@ def algorithmic_bytes(cfg) -> int:
 NCU_TRAFFIC = {
     ("umma", "c2"): {"bytes": 82.36e6,
                      "sources": ("paper_2304_04237_b200/csrc/umma_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
-                     "sha256": "fb6271a22b903eb5567462f4142ddce64afcce81976907746c5e9cec44ff4d94"},
+                     "sha256": "042004f8b9bd144905eb4965ebbbb8560f7b4e71dcef514804917616c539c08e"},
 }
 
 
@@ -214,7 +214,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
-    ap.add_argument("--variant", default="auto", choices=["auto", "direct", "mma", "mma_ws", "umma"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "direct", "mma", "mma_ws", "umma", "umma_ts"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -261,8 +261,8 @@ def main():
     ctx = sa.slide_attn_create(cfg["B"], cfg["H"], cfg["W"], cfg["heads"], cfg["head_dim"],
                                cfg["ksize"], td, cfg["has_bias"])
     if args.variant != "auto":
-        sa.slide_attn_set_variant(ctx, {"direct": 1, "mma": 2, "mma_ws": 3, "umma": 4}[args.variant])
-    variant = {1: "direct", 2: "mma", 3: "mma_ws", 4: "umma"}[sa.slide_attn_get_variant(ctx)]
+        sa.slide_attn_set_variant(ctx, {"direct": 1, "mma": 2, "mma_ws": 3, "umma": 4, "umma_ts": 5}[args.variant])
+    variant = {1: "direct", 2: "mma", 3: "mma_ws", 4: "umma", 5: "umma_ts"}[sa.slide_attn_get_variant(ctx)]
     launches = sa.slide_attn_launches_per_forward(ctx)
     stream = torch.cuda.current_stream()
 

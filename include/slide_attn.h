@@ -82,8 +82,11 @@ typedef enum {
     SLIDE_ATTN_VARIANT_MMA_WS  = 3,   /* same arithmetic, persistent warp-specialised schedule (key
                                          warps / value warps, 3-stage TMA ring, weights resident in
                                          registers, single launch); bf16, head_dim 32, ksize 3          */
-    SLIDE_ATTN_VARIANT_UMMA    = 4    /* MMA_WS with the value-side contraction on the 5th-generation
+    SLIDE_ATTN_VARIANT_UMMA    = 4,   /* MMA_WS with the value-side contraction on the 5th-generation
                                          tensor core (tcgen05.mma, accumulator in tensor memory);
+                                         bf16, head_dim 32, ksize 3                                     */
+    SLIDE_ATTN_VARIANT_UMMA_TS = 5    /* both contractions on tcgen05.mma with their A operands (the
+                                         q.k products, the softmax weights) held in tensor memory;
                                          bf16, head_dim 32, ksize 3                                     */
 } slide_attn_variant;
 

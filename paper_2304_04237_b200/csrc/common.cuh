@@ -56,4 +56,9 @@ bool umma_supports(slide_attn_dtype dtype, int head_dim, int ksize);
 cudaError_t umma_setup();
 cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
 
+// UMMA_TS variant: both contractions on tcgen05 with their A operands in tensor memory.
+bool umma_ts_supports(slide_attn_dtype dtype, int head_dim, int ksize);
+cudaError_t umma_ts_setup();
+cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
+
 }  // namespace slide_attn

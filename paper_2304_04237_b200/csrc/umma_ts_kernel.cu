@@ -1,0 +1,663 @@
+// UMMA_TS variant (bf16, head_dim 32, k = 3): BOTH contractions of the fused forward on the
+// 5th-generation tensor core (tcgen05.mma), each with its A operand in tensor memory, so neither the
+// q.k products nor the softmax weights pass through shared memory.
+//
+// Arithmetic (Eq. 2 with Eq. 12 inside; w = E + D, E the one-hot shift of Eq. 11):
+//   product warps   P[p,(t,c)] = q[p,c] k[p+off(t),c]   packed bf16 multiply -> tcgen05.st (TMEM)
+//   key MMA         L[p,n]     = sum_{t,c} P[p,(t,c)] Bk[(t,c),n]       tcgen05.mma, A from TMEM
+//                   n = 0..8: deformed part D_k of slot n;  n = 9..17: plain q.k sum of tap n-9
+//   product warps   logit[s] = (L[s] + L[9+s]) scale + bias[s];  e = exp2(logit - max)
+//                   (tcgen05.ld.32x32b: one thread holds all logits of one pixel, no shuffles)
+//                   A' row = e_hi | e_hi | e_lo | e8_hi e8_hi e8_lo 0..   -> tcgen05.st (TMEM)
+//   value MMA       D[p,(t,c)] = sum_k A'[p,k] Bv[k,(t,c)]  (+16 sum columns)   A from TMEM
+//   value warps     out[p,c] = (sum_t D[p,t,c] v[p+off(t),c]) / sum[p]
+//
+// Tensor memory (512 columns): two value-chunk slots of 112 (chunk c = 3 blk + dx -> slot c & 1), four
+// P chunks of 48 (3 taps x 32 bf16, chunk -> buffer c & 3), two logit tiles of 32, two A' tiles of 16.
+//
+// Warps (15): 0-7 value warps (quadrant = warp % 4, pixel-row pair = warp / 4, every block), 8-11
+// product warps (one per quadrant: P of block b, then the softmax of block b - 1), 12 and 14 key-side
+// control (K/q TMA; the 18 key MMAs of the even / odd blocks; chunks are claimed in order through one
+// shared word so that a P-ready barrier is only ever tested for its current or just completed
+// phase), 13 value-side control (V TMA, value MMAs).  Warp 12 owns tensor memory.  Every wait is
+// bounded; a wait that runs out sets the status word, and tensor memory is released on every path.
+//
+// Slower than the UMMA variant on the measured workloads (the key side needs 18 MMA instructions of
+// N = 32 per 128 pixels and every role pays a TMEM round trip per chunk); kept selectable for A/B.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace slide_attn {
+
+namespace {
+
+constexpr int kHeadDim = 32;
+constexpr int kVWarps = 8;
+constexpr int kPWarps = 4;
+constexpr int kCtlK = kVWarps + kPWarps;                // warp 12
+constexpr int kCtlV = kCtlK + 1;                        // warp 13
+constexpr int kCtlK2 = kCtlV + 1;                      // warp 14: key MMAs of the odd blocks
+constexpr int kThreads = (kCtlK2 + 1) * 32;             // 480
+constexpr int kKStages = 2;
+constexpr int kMaxVStages = 4;
+constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
+constexpr int kBBytes = kBCols * 64;
+constexpr int kBkBytes = 36 * 512;                      // key-side B: 288 K x 32 N bf16
+constexpr int kWeightBytes = kHeadDim * 81 * 4;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kTmemCols = 512;
+// tensor-memory columns
+constexpr uint32_t kColD = 0;                           // two value-chunk slots of 112 columns (chunk c -> slot c & 1)
+constexpr uint32_t kColP = 224;                         // four P chunks of 48 columns (3 taps x 32 bf16)
+constexpr uint32_t kColL = 416;                         // two logit tiles of 32 columns
+constexpr uint32_t kColE = 480;                         // two A' tiles of 16 columns (32 bf16)
+constexpr uint32_t kIdesc96 = umma_idesc_bf16(128, 96);
+constexpr uint32_t kIdesc112 = umma_idesc_bf16(128, 112);
+constexpr uint32_t kIdesc32 = umma_idesc_bf16(128, 32);
+
+struct UmmaParams {
+    const float* wk;
+    const float* wv;
+    const float* bias;
+    __nv_bfloat16* out;
+    int* status;
+    int B, H, W, heads;
+    int TW;
+    int tiles_x, tiles_y;
+    int stages;
+    float scale_log2e;
+};
+
+struct Smem {
+    uint32_t halo_pad, kstage_bytes, v_off, b_off, bk_off, tmem_off, bar_off, total;
+};
+
+__host__ __device__ inline Smem smem_layout(int TW, int vstages) {
+    Smem s;
+    s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 1023u) & ~1023u;
+    const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
+    if (s.halo_pad < wbytes) s.halo_pad = wbytes;
+    s.kstage_bytes = s.halo_pad + (((uint32_t)(4 * TW * 64) + 1023u) & ~1023u);
+    s.v_off = kKStages * s.kstage_bytes;
+    s.b_off = s.v_off + vstages * s.halo_pad;
+    s.bk_off = s.b_off + kBBytes;
+    s.tmem_off = s.bk_off + kBkBytes;
+    s.bar_off = s.tmem_off + 16;
+    s.total = s.bar_off + 40 * 8 + 1024;
+    return s;
+}
+
+constexpr int kBarKFull = 0;         // [2]
+constexpr int kBarKEmpty = 2;        // [2]  count 4
+constexpr int kBarVFull = 4;         // [4]
+constexpr int kBarVEmpty = 8;        // [4]  count 8
+constexpr int kBarWeights = 12;
+constexpr int kBarWeightsDone = 13;  // count 14
+constexpr int kBarPReady = 14;       // [4]  count 4: P chunk stored by the four product warps
+constexpr int kBarPFree = 18;        // [4]  key MMAs reading the chunk are complete
+constexpr int kBarLFull = 22;        // [2]  logits of a block complete
+constexpr int kBarLFree = 24;        // [2]  count 4: logits read
+constexpr int kBarEReady = 26;       // [2]  count 4: A' rows stored
+constexpr int kBarEFree = 28;        // [2]  value MMAs of the block complete
+constexpr int kBarDFull = 30;        // [2]  value chunk complete
+constexpr int kBarDFree = 32;        // [2]  count 8: value chunk read
+constexpr int kBarVDone = 34;        // count 8
+
+__device__ __forceinline__ uint4 lds_u4(const unsigned char* base, uint32_t off) {
+    return *reinterpret_cast<const uint4*>(base + off);
+}
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+             const __grid_constant__ CUtensorMap map_v, const UmmaParams P)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const Smem L = smem_layout(P.TW, P.stages);
+    const uint32_t bar0 = smem_u32(smem + L.bar_off);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tig = lane & 3;
+    const int SV = P.stages;
+    const int U = P.TW >> 3;
+    const int HW2 = P.TW + 2;
+
+    const int h = blockIdx.x % P.heads;
+    const int rank = blockIdx.x / P.heads;
+    const int nrank = ((int)gridDim.x - h + P.heads - 1) / P.heads;
+    const int tiles_per_head = P.B * P.tiles_y * P.tiles_x;
+    const int my_tiles = rank < tiles_per_head ? (tiles_per_head - rank + nrank - 1) / nrank : 0;
+    const int my_units = my_tiles * U;
+    const int my_blocks = (my_units + 3) >> 2;
+    const int C = P.heads * kHeadDim;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kKStages; ++s) { mbar_init(bar(kBarKFull + s), 1); mbar_init(bar(kBarKEmpty + s), kPWarps); }
+        for (int s = 0; s < kMaxVStages; ++s) { mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarVEmpty + s), kVWarps); }
+        mbar_init(bar(kBarWeights), 1);
+        mbar_init(bar(kBarWeightsDone), kThreads / 32);
+        for (int i = 0; i < 4; ++i) { mbar_init(bar(kBarPReady + i), kPWarps); mbar_init(bar(kBarPFree + i), 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(kBarLFull + i), 1);
+            mbar_init(bar(kBarLFree + i), kPWarps);
+            mbar_init(bar(kBarEReady + i), kPWarps);
+            mbar_init(bar(kBarEFree + i), 1);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(kBarDFull + i), 1); mbar_init(bar(kBarDFree + i), kVWarps); }
+        mbar_init(bar(kBarVDone), kVWarps);
+        *reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + 39 * 8) = 0u;
+    }
+    if (warp == kCtlK) tmem_alloc(smem_u32(smem + L.tmem_off), kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *reinterpret_cast<const volatile uint32_t*>(smem + L.tmem_off);
+
+    struct TileWalk { int tx, ty, b, stage, round; };
+    const int step_tx = nrank % P.tiles_x, step_ty = (nrank / P.tiles_x) % P.tiles_y,
+              step_b = nrank / (P.tiles_x * P.tiles_y);
+    auto walk_begin = [&]() {
+        TileWalk w;
+        w.tx = rank % P.tiles_x;
+        w.ty = (rank / P.tiles_x) % P.tiles_y;
+        w.b = rank / (P.tiles_x * P.tiles_y);
+        w.stage = 0; w.round = 0;
+        return w;
+    };
+    auto walk_next = [&](TileWalk& w, int nstages) {
+        w.tx += step_tx;
+        if (w.tx >= P.tiles_x) { w.tx -= P.tiles_x; ++w.ty; }
+        w.ty += step_ty;
+        if (w.ty >= P.tiles_y) { w.ty -= P.tiles_y; ++w.b; }
+        w.b += step_b;
+        if (++w.stage == nstages) { w.stage = 0; ++w.round; }
+    };
+    auto issue_k_tile = [&](const TileWalk& w) {
+        const uint32_t base = smem_u32(smem + (size_t)w.stage * L.kstage_bytes);
+        const uint32_t fb = bar(kBarKFull + w.stage);
+        mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64 + 4 * P.TW * 64));
+        tma_load_4d(base, &map_k, fb, h * kHeadDim, w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
+        tma_load_4d(base + L.halo_pad, &map_q, fb, h * kHeadDim, w.tx * P.TW, w.ty * 4, w.b);
+    };
+    auto issue_v_tile = [&](const TileWalk& w) {
+        const uint32_t fb = bar(kBarVFull + w.stage);
+        mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64));
+        tma_load_4d(smem_u32(smem + L.v_off + (size_t)w.stage * L.halo_pad), &map_v, fb, h * kHeadDim,
+                    w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
+    };
+
+    // weights staged in the last V stage; first K tiles and V tiles go out at once
+    const unsigned char* w_stage = smem + L.v_off + (size_t)(SV - 1) * L.halo_pad;
+    int k_issued = 0, v_issued = 0;
+    TileWalk kq = walk_begin(), vq = kq;
+    if (my_tiles > 0 && warp == kCtlK && lane == 0) {
+        mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
+        bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
+        bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
+        while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
+    }
+    if (my_tiles > 0 && warp == kCtlV && lane == 0) {
+        while (v_issued < my_tiles && v_issued < SV - 1) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
+    }
+    __syncwarp();
+
+    bool ok = my_tiles > 0 && warp_wait(bar(kBarWeights), 0);
+    const float* wks = reinterpret_cast<const float*>(w_stage);
+    const float* wvs = wks + kHeadDim * 81;
+
+    if (ok) {
+        // ---- value-side B tile: column n = (tap-column-major tap, channel), 64 bytes of K each --------
+        unsigned char* sB = smem + L.b_off;
+        for (int n = threadIdx.x; n < kBCols; n += kThreads) {
+            unsigned char* col = sB + (n >> 3) * 512 + (n & 7) * 16;
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i] = 0u;
+            if (n >= 288) {
+#pragma unroll
+                for (int i = 4; i < 12; ++i) w[i] = kOnesBf16x2;
+                w[12] = pack_bf16(0.f, 1.f); w[13] = pack_bf16(1.f, 0.f);
+            } else {
+                const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;
+                const int cn = n & 31, j = cn >> 3, wi = cn & 7;
+                const float* wc = wvs + (8 * (wi >> 1) + 2 * j + (wi & 1)) * 81 + t;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int s0 = 2 * i, s1 = 2 * i + 1;
+                    w[i] = pack_bf16(wc[s0 * 9] - (s0 == t ? 1.f : 0.f), wc[s1 * 9] - (s1 == t ? 1.f : 0.f));
+                    const uint32_t oh = pack_bf16(s0 == t ? 1.f : 0.f, s1 == t ? 1.f : 0.f);
+                    w[4 + i] = oh; w[8 + i] = oh;
+                }
+                const float o8 = t == 8 ? 1.f : 0.f;
+                w[12] = pack_bf16(wc[72] - o8, o8); w[13] = pack_bf16(o8, 0.f);
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4*>(col + c * 128) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+        }
+        // ---- key-side B: [k-group of 8][n-group of 8][8 n rows][8 k] bf16; K index = 32 tap + kappa,
+        // kappa -> channel as the product warps' tcgen05.st lays P out
+        unsigned char* sBk = smem + L.bk_off;
+        for (int item = threadIdx.x; item < 36 * 32; item += kThreads) {
+            const int n = item & 31, kg = item >> 5;
+            const int t = kg >> 2, kap0 = (kg & 3) * 8;
+            float val[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int kap = kap0 + e;
+                const int c = 8 * ((kap & 15) >> 2) + (kap & 3) + (kap >= 16 ? 4 : 0);
+                float x = 0.f;
+                if (n < 9) x = wks[c * 81 + n * 9 + t] - (n == t ? 1.f : 0.f);
+                else if (n < 18) x = (n - 9 == t) ? 1.f : 0.f;
+                val[e] = x;
+            }
+            *reinterpret_cast<uint4*>(sBk + kg * 512 + (n >> 3) * 128 + (n & 7) * 16) =
+                make_uint4(pack_bf16(val[0], val[1]), pack_bf16(val[2], val[3]), pack_bf16(val[4], val[5]), pack_bf16(val[6], val[7]));
+        }
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
+
+    if (warp >= kVWarps && warp < kCtlK) {
+        // =====================================================================================
+        // product warps: quadrant q of every block = unit 4 blk + q
+        // =====================================================================================
+        const int q = warp - kVWarps;                              // == warp % 4
+        const uint32_t tq = tmem + ((uint32_t)(32 * q) << 16);
+        float biasl[9];
+#pragma unroll
+        for (int s = 0; s < 9; ++s) biasl[s] = P.bias ? P.bias[h * 9 + s] * kLog2e : 0.f;
+
+        // softmax of block sb (thread = pixel = TMEM lane 32 q + lane); `valid`: the unit exists
+        auto softmax_block = [&](int sb, bool valid) -> bool {
+            const int lb = sb & 1;
+            if (!warp_wait(bar(kBarLFull + lb), (sb >> 1) & 1)) return false;
+            tc_fence_after_sync();
+            float Lg[32];
+            tmem_ld_32x32b_x32(tq + kColL + 32 * lb, Lg);
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarLFree + lb));
+            uint32_t row[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) row[i] = 0u;
+            if (valid) {
+                float l[9], m = -INFINITY;
+#pragma unroll
+                for (int s = 0; s < 9; ++s) { l[s] = (Lg[s] + Lg[9 + s]) * P.scale_log2e + biasl[s]; m = fmaxf(m, l[s]); }
+                float hi[9], lo[9];
+#pragma unroll
+                for (int s = 0; s < 9; ++s) {
+                    const float e = fast_exp2(l[s] - m);
+                    hi[s] = __bfloat162float(__float2bfloat16_rn(e));
+                    lo[s] = e - hi[s];
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    row[i] = pack_bf16(hi[2 * i], hi[2 * i + 1]);
+                    row[4 + i] = row[i];
+                    row[8 + i] = pack_bf16(lo[2 * i], lo[2 * i + 1]);
+                }
+                row[12] = pack_bf16(hi[8], hi[8]);
+                row[13] = pack_bf16(lo[8], 0.f);
+            }
+            if (!warp_wait(bar(kBarEFree + lb), ((sb >> 1) & 1) ^ 1)) return false;
+            tc_fence_after_sync();
+            tmem_st_32x32b_x16(tq + kColE + 16 * lb, row);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarEReady + lb));
+            return true;
+        };
+
+        int done_blocks = 0;                                       // blocks whose P this warp has delivered
+        for (int ti = 0; ok && ti < my_tiles; ++ti) {
+            const int stage = ti % kKStages;
+            if (!warp_wait(bar(kBarKFull + stage), (ti / kKStages) & 1)) { ok = false; break; }
+            const int u0 = ti * U;
+            for (int ul = (q + 4 - u0 % 4) % 4; ul < U; ul += 4) {
+                const int u = u0 + ul, blk = u >> 2;
+                const int ux = ul * 8;
+                const unsigned char* sK = smem + (size_t)stage * L.kstage_bytes;
+                const unsigned char* sQ = sK + L.halo_pad;
+                uint32_t qf[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 v = lds_u4(sQ, (uint32_t)(i * P.TW + ux + g) * 64u + tig * 16u);
+                    qf[i][0] = v.x; qf[i][1] = v.y; qf[i][2] = v.z; qf[i][3] = v.w;
+                }
+                const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
+#pragma unroll
+                for (int dx = 0; dx < 3; ++dx) {
+                    const int pc = 3 * blk + dx, pb = pc & 3;
+                    uint4 kc[6];
+#pragma unroll
+                    for (int r = 0; r < 6; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)(r * HW2 + dx) * 64u);
+                    if (!warp_wait(bar(kBarPFree + pb), ((pc >> 2) & 1) ^ 1)) { ok = false; break; }
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy) {
+#pragma unroll
+                        for (int mt = 0; mt < 2; ++mt) {
+                            const uint4 k0 = kc[2 * mt + dy], k1 = kc[2 * mt + dy + 1];   // pixel rows 2mt / 2mt+1
+                            uint32_t r[8];
+                            r[0] = hmul2_bf16(qf[2 * mt][0], k0.x);     r[1] = hmul2_bf16(qf[2 * mt][1], k0.y);
+                            r[2] = hmul2_bf16(qf[2 * mt + 1][0], k1.x); r[3] = hmul2_bf16(qf[2 * mt + 1][1], k1.y);
+                            r[4] = hmul2_bf16(qf[2 * mt][2], k0.z);     r[5] = hmul2_bf16(qf[2 * mt][3], k0.w);
+                            r[6] = hmul2_bf16(qf[2 * mt + 1][2], k1.z); r[7] = hmul2_bf16(qf[2 * mt + 1][3], k1.w);
+                            tmem_st_16x256b_x2(tq + ((uint32_t)(16 * mt) << 16) + kColP + 48 * pb + 16 * dy, r);
+                        }
+                    }
+                    tmem_wait_st();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarPReady + pb));
+                }
+                if (!ok) break;
+                ++done_blocks;
+                // the logits of the block before are complete by now (or soon)
+                if (blk > 0 && !softmax_block(blk - 1, true)) { ok = false; break; }
+            }
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(bar(kBarKEmpty + stage));
+        }
+        // a quadrant the last block lacks: deliver its (empty) share so that the counts complete
+        if (ok && done_blocks < my_blocks) {
+            const int blk = my_blocks - 1;
+            for (int dx = 0; ok && dx < 3; ++dx) {
+                const int pc = 3 * blk + dx, pb = pc & 3;
+                if (!warp_wait(bar(kBarPFree + pb), ((pc >> 2) & 1) ^ 1)) { ok = false; break; }
+                if (lane == 0) mbar_arrive(bar(kBarPReady + pb));
+            }
+            if (ok && blk > 0 && !softmax_block(blk - 1, true)) ok = false;
+            if (ok && !softmax_block(blk, false)) ok = false;
+        } else if (ok && my_blocks > 0) {
+            if (!softmax_block(my_blocks - 1, true)) ok = false;
+        }
+    } else if (warp < kVWarps) {
+        // =====================================================================================
+        // value warps: warp (qd, m) takes pixel rows 2m, 2m+1 of quadrant qd of every block
+        // =====================================================================================
+        const int qd = warp & 3, m = warp >> 2;
+        const uint32_t tq = tmem + ((uint32_t)(32 * qd + 16 * m) << 16);
+
+        TileWalk vw = walk_begin();
+        for (int ti = 0; ok && ti < my_tiles; ++ti, walk_next(vw, SV)) {
+            const int tx = vw.tx, ty = vw.ty, b = vw.b, stage = vw.stage;
+            if (!warp_wait(bar(kBarVFull + stage), vw.round & 1)) { ok = false; break; }
+            const int u0 = ti * U;
+          for (int ul = (qd + 4 - u0 % 4) % 4; ul < U; ul += 4) {
+            const int u = u0 + ul;
+            const int ux = ul * 8;
+            const int blk = u >> 2;
+            const unsigned char* sV = smem + L.v_off + (size_t)stage * L.halo_pad;
+            const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
+
+            float o_acc[2][8];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) o_acc[i][c] = 0.f;
+            float inv[2] = {0.f, 0.f};
+
+#pragma unroll
+            for (int dx = 0; dx < 3; ++dx) {
+                const int cs = 3 * blk + dx, ds = cs & 1;
+                if (!warp_wait(bar(kBarDFull + ds), (cs >> 1) & 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t colbase = kColD + ds * 112;
+                {
+                    uint32_t dr[48];
+                    const uint32_t ta = tq + colbase;
+                    tmem_ld3_16x256b_x4_nowait(ta, ta + 32, ta + 64, dr);
+                    uint4 vp[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) vp[r] = lds_u4(sV, off0 + (uint32_t)((2 * m + r) * HW2 + dx) * 64u);
+                    float vf[4][8];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const uint4 v = vp[r];
+                        vf[r][0] = bf16_lo(v.x); vf[r][1] = bf16_hi(v.x);
+                        vf[r][2] = bf16_lo(v.y); vf[r][3] = bf16_hi(v.y);
+                        vf[r][4] = bf16_lo(v.z); vf[r][5] = bf16_hi(v.z);
+                        vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
+                    }
+                    tmem_wait_ld48(dr);
+                    float d[48];
+#pragma unroll
+                    for (int i = 0; i < 48; ++i) d[i] = __uint_as_float(dr[i]);
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            ffma2(o_acc[0][2 * j], o_acc[0][2 * j + 1], d[16 * dy + 4 * j], d[16 * dy + 4 * j + 1],
+                                  vf[dy][2 * j], vf[dy][2 * j + 1]);
+                            ffma2(o_acc[1][2 * j], o_acc[1][2 * j + 1], d[16 * dy + 4 * j + 2], d[16 * dy + 4 * j + 3],
+                                  vf[dy + 1][2 * j], vf[dy + 1][2 * j + 1]);
+                        }
+                    }
+                }
+                if (dx == 2) {
+                    float s0[4];
+                    tmem_ld_16x256b_x1(tq + colbase + 96, s0);
+                    inv[0] = rcp_approx(s0[0]); inv[1] = rcp_approx(s0[2]);
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
+            }
+            if (!ok) break;
+
+            {
+                const int x = tx * P.TW + ux + g, y0 = ty * 4 + 2 * m;
+                __nv_bfloat16* op = P.out + ((size_t)(b * P.H + y0) * P.W + x) * C + h * kHeadDim + tig * 8;
+                const size_t row_stride = (size_t)P.W * C;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    if (x < P.W && y0 + i < P.H) {
+                        uint4 r;
+                        r.x = pack_bf16(o_acc[i][0] * inv[i], o_acc[i][1] * inv[i]);
+                        r.y = pack_bf16(o_acc[i][2] * inv[i], o_acc[i][3] * inv[i]);
+                        r.z = pack_bf16(o_acc[i][4] * inv[i], o_acc[i][5] * inv[i]);
+                        r.w = pack_bf16(o_acc[i][6] * inv[i], o_acc[i][7] * inv[i]);
+                        *reinterpret_cast<uint4*>(op + i * row_stride) = r;
+                    }
+                }
+            }
+          }
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(bar(kBarVEmpty + stage));
+        }
+        // quadrants of the last block that hold no unit: keep the chunk barriers in step
+        if (ok && my_blocks > 0 && (my_units & 3) != 0 && qd >= (my_units & 3)) {
+            for (int dx = 0; ok && dx < 3; ++dx) {
+                const int cs = 3 * (my_blocks - 1) + dx, ds = cs & 1;
+                if (!warp_wait(bar(kBarDFull + ds), (cs >> 1) & 1)) { ok = false; break; }
+                if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
+            }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kBarVDone));
+    } else if (warp == kCtlK || warp == kCtlK2) {
+        // =====================================================================================
+        // key-side control: K/q tiles (warp 12) and the key MMAs (18 per block: 9 taps x two K = 16
+        // halves); warp 12 takes the even blocks, warp 14 the odd ones.  Chunks are CLAIMED in order
+        // through one word, so a P-ready barrier is only ever tested for its current or its just
+        // completed phase; the MMAs themselves go out side by side.
+        // =====================================================================================
+        if (lane == 0 && ok) {
+            const uint32_t sBk0 = smem_u32(smem + L.bk_off);
+            volatile uint32_t* claim = reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + 39 * 8);
+            const bool first = warp == kCtlK;
+            int blk = first ? 0 : 1, dx = 0;
+            const int my_k_tiles = first ? my_tiles - k_issued : 0;
+            const int my_k_blocks = first ? (my_blocks + 1) / 2 : my_blocks / 2;
+            int left = my_k_tiles + 3 * my_k_blocks;
+            uint32_t idle = 0;
+            while (left > 0) {
+                const int pc = 3 * blk + dx, pb = pc & 3, lb = blk & 1;
+                const uint32_t tK = mbar_test_u32(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1);
+                const uint32_t tL = mbar_test_u32(bar(kBarLFree + lb), ((blk >> 1) & 1) ^ 1);
+                const bool my_turn = blk < my_blocks && *claim == (uint32_t)pc;
+                const uint32_t tP = my_turn ? mbar_test_u32(bar(kBarPReady + pb), (pc >> 2) & 1) : 0u;
+                const int left_before = left;
+                if (first && tK != 0 && k_issued < my_tiles) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; --left; }
+                if (tP != 0 && (dx != 0 || tL != 0)) {
+                    *claim = (uint32_t)pc + 1u;
+                    tc_fence_after_sync();
+                    const uint32_t dcol = tmem + kColL + 32 * lb;
+                    const uint32_t acol = tmem + kColP + 48 * pb;
+                    const uint32_t bdx = sBk0 + (uint32_t)dx * 4u * 512u;
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy) {
+#pragma unroll
+                        for (int kh = 0; kh < 2; ++kh)
+                            umma_bf16_ts(dcol, acol + 16 * dy + 8 * kh,
+                                         umma_smem_desc(bdx + (uint32_t)(dy * 12 + kh * 2) * 512u, 512, 128),
+                                         kIdesc32, (dx != 0 || dy != 0 || kh != 0) ? 1u : 0u);
+                    }
+                    umma_commit(bar(kBarPFree + pb));
+                    if (dx == 2) { umma_commit(bar(kBarLFull + lb)); dx = 0; blk += 2; }
+                    else ++dx;
+                    --left;
+                }
+                if (left != left_before) idle = 0;
+                else if (++idle > (1u << 24)) { ok = false; break; }
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (warp == kCtlK) {
+            if (my_tiles > 0 && !warp_wait(bar(kBarVDone), 0)) ok = false;
+            tc_fence_after_sync();
+            __syncwarp();
+            tmem_dealloc(tmem, kTmemCols);
+        }
+    } else {
+        // =====================================================================================
+        // value-side control: V tiles and the value MMAs (chunk dx of block blk -> TMEM slot dx)
+        // =====================================================================================
+        if (lane == 0 && ok) {
+            const uint32_t sB0 = smem_u32(smem + L.b_off);
+            bool weights_done = false;
+            int blk = 0, dx = 0;
+            int left = my_tiles - v_issued + 3 * my_blocks;
+            uint32_t idle = 0;
+            while (left > 0) {
+                if (!weights_done) weights_done = mbar_test(bar(kBarWeightsDone), 0);
+                const int eb = blk & 1;
+                const uint32_t tV = mbar_test_u32(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
+                const uint32_t tE = mbar_test_u32(bar(kBarEReady + eb), (blk >> 1) & 1);
+                const int cs = 3 * blk + dx, ds = cs & 1;
+                const uint32_t tD = mbar_test_u32(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1);
+                const int left_before = left;
+                if (tV != 0 && v_issued < my_tiles && (v_issued != SV - 1 || weights_done)) {
+                    issue_v_tile(vq); walk_next(vq, SV); ++v_issued; --left;
+                }
+                if (blk < my_blocks && tE != 0 && tD != 0) {
+                    tc_fence_after_sync();
+                    const uint32_t sB = sB0 + dx * 12 * 512;
+                    const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
+                    const uint32_t dcol = tmem + kColD + ds * 112;
+                    const uint32_t acol = tmem + kColE + 16 * eb;
+                    umma_bf16_ts(dcol, acol, umma_smem_desc(sB, 128, 512), idesc, 0);
+                    umma_bf16_ts(dcol, acol + 8, umma_smem_desc(sB + 256, 128, 512), idesc, 1);
+                    umma_commit(bar(kBarDFull + ds));
+                    if (dx == 2) { umma_commit(bar(kBarEFree + eb)); dx = 0; ++blk; }
+                    else ++dx;
+                    --left;
+                }
+                if (left != left_before) idle = 0;
+                else if (++idle > (1u << 24)) { ok = false; break; }
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    }
+    if (!ok && my_tiles > 0 && lane == 0) atomicExch(P.status, 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+bool make_map(CUtensorMap* map, const void* base, int B, int H, int W, int C, int bw, int bh) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)bw, (cuuint32_t)bh, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t kMaxSmem = 227 * 1024;
+
+}  // namespace
+
+bool umma_ts_supports(slide_attn_dtype dtype, int head_dim, int ksize) {
+    return dtype == SLIDE_ATTN_BF16 && head_dim == kHeadDim && ksize == 3;
+}
+
+cudaError_t umma_ts_setup() {
+    if (!encode_fn()) return cudaErrorNotSupported;
+    return cudaFuncSetAttribute(umma_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+}
+
+cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStream_t stream) {
+    const int txn = (p.W + 63) / 64;
+    const int TW = ((((p.W + txn - 1) / txn) + 7) / 8) * 8;
+    UmmaParams P;
+    P.wk = p.wk; P.wv = p.wv; P.bias = p.bias;
+    P.out = static_cast<__nv_bfloat16*>(p.out);
+    P.status = d_status;
+    P.B = p.B; P.H = p.H; P.W = p.W; P.heads = p.heads;
+    P.TW = TW;
+    P.tiles_x = (p.W + TW - 1) / TW;
+    P.tiles_y = (p.H + 3) / 4;
+    P.stages = 2;
+    for (int st = kMaxVStages; st >= 2; --st)
+        if (smem_layout(TW, st).total <= kMaxSmem) { P.stages = st; break; }
+    P.scale_log2e = kLog2e / sqrtf((float)kHeadDim);
+    const Smem L = smem_layout(TW, P.stages);
+    if (L.total > kMaxSmem) return cudaErrorInvalidConfiguration;
+
+    const int C = p.heads * kHeadDim;
+    CUtensorMap map_q, map_k, map_v;
+    if (!make_map(&map_q, p.q, p.B, p.H, p.W, C, TW, 4) ||
+        !make_map(&map_k, p.k, p.B, p.H, p.W, C, TW + 2, 6) ||
+        !make_map(&map_v, p.v, p.B, p.H, p.W, C, TW + 2, 6))
+        return cudaErrorInvalidValue;
+
+    const long long tiles = (long long)P.tiles_x * P.tiles_y * p.B * p.heads;
+    if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    int grid = num_sms;
+    if (grid < p.heads) grid = p.heads;
+    if ((long long)grid > tiles) grid = (int)tiles;
+    umma_ts_kernel<<<grid, kThreads, L.total, stream>>>(map_q, map_k, map_v, P);
+    return cudaGetLastError();
+}
+
+}  // namespace slide_attn

@@ -15,7 +15,7 @@ from util import TORCH_DTYPE, VARIANTS, assert_close, gpu_forward, to_device
 
 pytestmark = pytest.mark.gpu
 
-ALL_VARIANTS = ["auto", "direct", "mma", "mma_ws", "umma"]
+ALL_VARIANTS = ["auto", "direct", "mma", "mma_ws", "umma", "umma_ts"]
 
 
 def ref_forward(x, k):
@@ -198,7 +198,7 @@ def test_deterministic_and_leaves_guard_bands_alone(variant):
         sa.slide_attn_destroy(ctx)
 
 
-@pytest.mark.parametrize("variant", ["mma_ws", "umma"])
+@pytest.mark.parametrize("variant", ["mma_ws", "umma", "umma_ts"])
 def test_pipelined_variants_many_shapes_repeatable(variant):
     """The persistent kernels hand work between warps through mbarrier rings; shapes with many or
     few tiles per CTA, partial last blocks and ragged widths must all give the DIRECT variant's

@@ -44,7 +44,7 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
 }
 
 slide_attn_variant pick_variant(const slide_attn_ctx* c) {
-    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA, SLIDE_ATTN_VARIANT_MMA_WS,
+    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA_TS, SLIDE_ATTN_VARIANT_UMMA, SLIDE_ATTN_VARIANT_MMA_WS,
                                         SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_DIRECT};
     for (slide_attn_variant v : order)
         if (variant_supported(c, v)) return v;

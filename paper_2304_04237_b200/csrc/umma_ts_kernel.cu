@@ -15,15 +15,20 @@
 // Tensor memory (512 columns): two value-chunk slots of 112 (chunk c = 3 blk + dx -> slot c & 1), four
 // P chunks of 48 (3 taps x 32 bf16, chunk -> buffer c & 3), two logit tiles of 32, two A' tiles of 16.
 //
-// Warps (15): 0-7 value warps (quadrant = warp % 4, pixel-row pair = warp / 4, every block), 8-11
-// product warps (one per quadrant: P of block b, then the softmax of block b - 1), 12 and 14 key-side
-// control (K/q TMA; the 18 key MMAs of the even / odd blocks; chunks are claimed in order through one
-// shared word so that a P-ready barrier is only ever tested for its current or just completed
-// phase), 13 value-side control (V TMA, value MMAs).  Warp 12 owns tensor memory.  Every wait is
-// bounded; a wait that runs out sets the status word, and tensor memory is released on every path.
+// Warps (20, 93 registers): 0-7 value warps (quadrant = warp % 4, pixel-row pair = warp / 4, every
+// block), 8-15 product warps (quadrant, pixel-row pair: P of their 16 pixels of every block; the
+// softmax of a block is done for the whole quadrant by the warp whose pair index equals the block's
+// parity, after it has stored the P of the next block), 16 and 18 key-side control (the 18 key MMAs
+// of the even / odd blocks, taking turns through two barriers so that the P-ready barriers are
+// waited on strictly in chunk order), 17 value-side control
+// (value MMAs), 19 TMA thread (K/q and V rings).  The MMA threads have one thing to wait for at a
+// time and park in mbarrier waits instead of polling: that alone was worth 10 % of the kernel time.
+// Warp 16 owns tensor memory.  Every wait is bounded; a wait that runs out sets the status word, and
+// tensor memory is released on every path.
 //
-// Slower than the UMMA variant on the measured workloads (the key side needs 18 MMA instructions of
-// N = 32 per 128 pixels and every role pays a TMEM round trip per chunk); kept selectable for A/B.
+// What bounds it: the tensor pipe takes about 85 cycles per MMA instruction however small
+// (18 of N = 32 and 6 of N = 96 / 112 per 128 pixels, 2.2 k cycles), the value warps need about as
+// long per block, and the measured block period is 2.9 k cycles.
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -33,11 +38,12 @@ namespace {
 
 constexpr int kHeadDim = 32;
 constexpr int kVWarps = 8;
-constexpr int kPWarps = 4;
-constexpr int kCtlK = kVWarps + kPWarps;                // warp 12
-constexpr int kCtlV = kCtlK + 1;                        // warp 13
-constexpr int kCtlK2 = kCtlV + 1;                      // warp 14: key MMAs of the odd blocks
-constexpr int kThreads = (kCtlK2 + 1) * 32;             // 480
+constexpr int kPWarps = 8;
+constexpr int kCtlK = kVWarps + kPWarps;                // warp 16: key MMAs of the even blocks, TMEM owner
+constexpr int kCtlV = kCtlK + 1;                        // warp 17: value MMAs
+constexpr int kCtlK2 = kCtlV + 1;                       // warp 18: key MMAs of the odd blocks
+constexpr int kCtlT = kCtlK2 + 1;                       // warp 19: TMA thread, K/q and V tiles
+constexpr int kThreads = (kCtlT + 1) * 32;
 constexpr int kKStages = 2;
 constexpr int kMaxVStages = 4;
 constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
@@ -88,20 +94,21 @@ __host__ __device__ inline Smem smem_layout(int TW, int vstages) {
 }
 
 constexpr int kBarKFull = 0;         // [2]
-constexpr int kBarKEmpty = 2;        // [2]  count 4
+constexpr int kBarKEmpty = 2;        // [2]  count 8 (product warps)
 constexpr int kBarVFull = 4;         // [4]
 constexpr int kBarVEmpty = 8;        // [4]  count 8
 constexpr int kBarWeights = 12;
-constexpr int kBarWeightsDone = 13;  // count 14
-constexpr int kBarPReady = 14;       // [4]  count 4: P chunk stored by the four product warps
+constexpr int kBarWeightsDone = 13;  // count 20 (every warp)
+constexpr int kBarPReady = 14;       // [4]  count 8: P chunk stored by the eight product warps
 constexpr int kBarPFree = 18;        // [4]  key MMAs reading the chunk are complete
 constexpr int kBarLFull = 22;        // [2]  logits of a block complete
-constexpr int kBarLFree = 24;        // [2]  count 4: logits read
+constexpr int kBarLFree = 24;        // [2]  count 4: logits read (one product warp per quadrant)
 constexpr int kBarEReady = 26;       // [2]  count 4: A' rows stored
 constexpr int kBarEFree = 28;        // [2]  value MMAs of the block complete
 constexpr int kBarDFull = 30;        // [2]  value chunk complete
 constexpr int kBarDFree = 32;        // [2]  count 8: value chunk read
 constexpr int kBarVDone = 34;        // count 8
+constexpr int kBarTurn = 35;         // [2]  the other key-control thread has taken the last chunk of its block
 
 __device__ __forceinline__ uint4 lds_u4(const unsigned char* base, uint32_t off) {
     return *reinterpret_cast<const uint4*>(base + off);
@@ -143,13 +150,14 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int i = 0; i < 4; ++i) { mbar_init(bar(kBarPReady + i), kPWarps); mbar_init(bar(kBarPFree + i), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kBarLFull + i), 1);
-            mbar_init(bar(kBarLFree + i), kPWarps);
-            mbar_init(bar(kBarEReady + i), kPWarps);
+            mbar_init(bar(kBarLFree + i), 4);
+            mbar_init(bar(kBarEReady + i), 4);
             mbar_init(bar(kBarEFree + i), 1);
         }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(kBarDFull + i), 1); mbar_init(bar(kBarDFree + i), kVWarps); }
         mbar_init(bar(kBarVDone), kVWarps);
-        *reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + 39 * 8) = 0u;
+        mbar_init(bar(kBarTurn + 0), 1);
+        mbar_init(bar(kBarTurn + 1), 1);
     }
     if (warp == kCtlK) tmem_alloc(smem_u32(smem + L.tmem_off), kTmemCols);
     tc_fence_before_sync();
@@ -198,9 +206,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
         bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
         bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
-        while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
     }
-    if (my_tiles > 0 && warp == kCtlV && lane == 0) {
+    if (my_tiles > 0 && warp == kCtlT && lane == 0) {
+        while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
         while (v_issued < my_tiles && v_issued < SV - 1) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
     }
     __syncwarp();
@@ -268,7 +276,8 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // =====================================================================================
         // product warps: quadrant q of every block = unit 4 blk + q
         // =====================================================================================
-        const int q = warp - kVWarps;                              // == warp % 4
+        const int q = (warp - kVWarps) & 3;                        // == warp % 4
+        const int pm = (warp - kVWarps) >> 2;                      // pixel-row pair of the unit; softmax of blocks = pm mod 2
         const uint32_t tq = tmem + ((uint32_t)(32 * q) << 16);
         float biasl[9];
 #pragma unroll
@@ -318,6 +327,15 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         };
 
         int done_blocks = 0;                                       // blocks whose P this warp has delivered
+        int next_sm = pm;                                          // next block whose softmax is this warp's
+        // softmax of this warp's blocks below `upto`
+        auto softmax_upto = [&](int upto) -> bool {
+            while (next_sm < upto) {
+                if (!softmax_block(next_sm, 4 * next_sm + q < my_units)) return false;
+                next_sm += 2;
+            }
+            return true;
+        };
         for (int ti = 0; ok && ti < my_tiles; ++ti) {
             const int stage = ti % kKStages;
             if (!warp_wait(bar(kBarKFull + stage), (ti / kKStages) & 1)) { ok = false; break; }
@@ -327,33 +345,30 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const int ux = ul * 8;
                 const unsigned char* sK = smem + (size_t)stage * L.kstage_bytes;
                 const unsigned char* sQ = sK + L.halo_pad;
-                uint32_t qf[4][4];
+                uint32_t qf[2][4];                                 // pixel rows 2pm, 2pm+1 of column ux + g
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 v = lds_u4(sQ, (uint32_t)(i * P.TW + ux + g) * 64u + tig * 16u);
+                for (int i = 0; i < 2; ++i) {
+                    const uint4 v = lds_u4(sQ, (uint32_t)((2 * pm + i) * P.TW + ux + g) * 64u + tig * 16u);
                     qf[i][0] = v.x; qf[i][1] = v.y; qf[i][2] = v.z; qf[i][3] = v.w;
                 }
                 const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
 #pragma unroll
                 for (int dx = 0; dx < 3; ++dx) {
                     const int pc = 3 * blk + dx, pb = pc & 3;
-                    uint4 kc[6];
+                    uint4 kc[4];                                   // halo rows 2pm .. 2pm+3 of column dx
 #pragma unroll
-                    for (int r = 0; r < 6; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)(r * HW2 + dx) * 64u);
+                    for (int r = 0; r < 4; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)((2 * pm + r) * HW2 + dx) * 64u);
                     if (!warp_wait(bar(kBarPFree + pb), ((pc >> 2) & 1) ^ 1)) { ok = false; break; }
                     tc_fence_after_sync();
 #pragma unroll
                     for (int dy = 0; dy < 3; ++dy) {
-#pragma unroll
-                        for (int mt = 0; mt < 2; ++mt) {
-                            const uint4 k0 = kc[2 * mt + dy], k1 = kc[2 * mt + dy + 1];   // pixel rows 2mt / 2mt+1
-                            uint32_t r[8];
-                            r[0] = hmul2_bf16(qf[2 * mt][0], k0.x);     r[1] = hmul2_bf16(qf[2 * mt][1], k0.y);
-                            r[2] = hmul2_bf16(qf[2 * mt + 1][0], k1.x); r[3] = hmul2_bf16(qf[2 * mt + 1][1], k1.y);
-                            r[4] = hmul2_bf16(qf[2 * mt][2], k0.z);     r[5] = hmul2_bf16(qf[2 * mt][3], k0.w);
-                            r[6] = hmul2_bf16(qf[2 * mt + 1][2], k1.z); r[7] = hmul2_bf16(qf[2 * mt + 1][3], k1.w);
-                            tmem_st_16x256b_x2(tq + ((uint32_t)(16 * mt) << 16) + kColP + 48 * pb + 16 * dy, r);
-                        }
+                        const uint4 k0 = kc[dy], k1 = kc[dy + 1];
+                        uint32_t r[8];
+                        r[0] = hmul2_bf16(qf[0][0], k0.x); r[1] = hmul2_bf16(qf[0][1], k0.y);
+                        r[2] = hmul2_bf16(qf[1][0], k1.x); r[3] = hmul2_bf16(qf[1][1], k1.y);
+                        r[4] = hmul2_bf16(qf[0][2], k0.z); r[5] = hmul2_bf16(qf[0][3], k0.w);
+                        r[6] = hmul2_bf16(qf[1][2], k1.z); r[7] = hmul2_bf16(qf[1][3], k1.w);
+                        tmem_st_16x256b_x2(tq + ((uint32_t)(16 * pm) << 16) + kColP + 48 * pb + 16 * dy, r);
                     }
                     tmem_wait_st();
                     tc_fence_before_sync();
@@ -362,8 +377,8 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
                 if (!ok) break;
                 ++done_blocks;
-                // the logits of the block before are complete by now (or soon)
-                if (blk > 0 && !softmax_block(blk - 1, true)) { ok = false; break; }
+                // the logits of the blocks before this one are complete by now (or soon)
+                if (!softmax_upto(blk)) { ok = false; break; }
             }
             __syncwarp();
             if (ok && lane == 0) mbar_arrive(bar(kBarKEmpty + stage));
@@ -376,11 +391,8 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 if (!warp_wait(bar(kBarPFree + pb), ((pc >> 2) & 1) ^ 1)) { ok = false; break; }
                 if (lane == 0) mbar_arrive(bar(kBarPReady + pb));
             }
-            if (ok && blk > 0 && !softmax_block(blk - 1, true)) ok = false;
-            if (ok && !softmax_block(blk, false)) ok = false;
-        } else if (ok && my_blocks > 0) {
-            if (!softmax_block(my_blocks - 1, true)) ok = false;
         }
+        if (ok && !softmax_upto(my_blocks)) ok = false;
     } else if (warp < kVWarps) {
         // =====================================================================================
         // value warps: warp (qd, m) takes pixel rows 2m, 2m+1 of quadrant qd of every block
@@ -495,42 +507,36 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // =====================================================================================
         if (lane == 0 && ok) {
             const uint32_t sBk0 = smem_u32(smem + L.bk_off);
-            volatile uint32_t* claim = reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + 39 * 8);
-            const bool first = warp == kCtlK;
-            int blk = first ? 0 : 1, dx = 0;
-            const int my_k_tiles = first ? my_tiles - k_issued : 0;
-            const int my_k_blocks = first ? (my_blocks + 1) / 2 : my_blocks / 2;
-            int left = my_k_tiles + 3 * my_k_blocks;
-            uint32_t idle = 0;
-            while (left > 0) {
-                const int pc = 3 * blk + dx, pb = pc & 3, lb = blk & 1;
-                const uint32_t tK = mbar_test_u32(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1);
-                const uint32_t tL = mbar_test_u32(bar(kBarLFree + lb), ((blk >> 1) & 1) ^ 1);
-                const bool my_turn = blk < my_blocks && *claim == (uint32_t)pc;
-                const uint32_t tP = my_turn ? mbar_test_u32(bar(kBarPReady + pb), (pc >> 2) & 1) : 0u;
-                const int left_before = left;
-                if (first && tK != 0 && k_issued < my_tiles) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; --left; }
-                if (tP != 0 && (dx != 0 || tL != 0)) {
-                    *claim = (uint32_t)pc + 1u;
+            // This thread has one thing to wait for at a time, so it parks in the waits (bounded).
+            // The two threads take the blocks in turn: a thread starts block b only when the other
+            // one has got past the P-ready wait of the last chunk of block b - 1, so the P-ready
+            // barriers are waited on strictly in chunk order.
+            const int me = warp == kCtlK ? 0 : 1;
+            for (int blk = me, n = 0; ok && blk < my_blocks; blk += 2, ++n) {
+                const int lb = blk & 1;
+                const uint32_t dcol = tmem + kColL + 32 * lb;
+                // even blocks wait for the odd block before (none before block 0: parity 1 of a
+                // fresh barrier tests true), odd blocks for the even block before
+                if (!mbar_wait(bar(kBarTurn + me), me == 0 ? (uint32_t)((n - 1) & 1) : (uint32_t)(n & 1))) { ok = false; break; }
+                if (!mbar_wait(bar(kBarLFree + lb), ((blk >> 1) & 1) ^ 1)) { ok = false; break; }
+#pragma unroll
+                for (int dx = 0; dx < 3; ++dx) {
+                    const int pc = 3 * blk + dx, pb = pc & 3;
+                    if (!mbar_wait(bar(kBarPReady + pb), (pc >> 2) & 1)) { ok = false; break; }
+                    if (dx == 2) mbar_arrive(bar(kBarTurn + (me ^ 1)));
                     tc_fence_after_sync();
-                    const uint32_t dcol = tmem + kColL + 32 * lb;
                     const uint32_t acol = tmem + kColP + 48 * pb;
-                    const uint32_t bdx = sBk0 + (uint32_t)dx * 4u * 512u;
+                    const uint64_t bdesc = umma_smem_desc(sBk0 + (uint32_t)dx * 4u * 512u, 512, 128);
 #pragma unroll
                     for (int dy = 0; dy < 3; ++dy) {
 #pragma unroll
-                        for (int kh = 0; kh < 2; ++kh)
-                            umma_bf16_ts(dcol, acol + 16 * dy + 8 * kh,
-                                         umma_smem_desc(bdx + (uint32_t)(dy * 12 + kh * 2) * 512u, 512, 128),
+                        for (int kh = 0; kh < 2; ++kh)      // 16 bytes of descriptor address = 1 unit
+                            umma_bf16_ts(dcol, acol + 16 * dy + 8 * kh, bdesc + (uint64_t)((dy * 12 + kh * 2) * 32),
                                          kIdesc32, (dx != 0 || dy != 0 || kh != 0) ? 1u : 0u);
                     }
                     umma_commit(bar(kBarPFree + pb));
-                    if (dx == 2) { umma_commit(bar(kBarLFull + lb)); dx = 0; blk += 2; }
-                    else ++dx;
-                    --left;
+                    if (dx == 2) umma_commit(bar(kBarLFull + lb));
                 }
-                if (left != left_before) idle = 0;
-                else if (++idle > (1u << 24)) { ok = false; break; }
             }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -540,42 +546,56 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             __syncwarp();
             tmem_dealloc(tmem, kTmemCols);
         }
-    } else {
+    } else if (warp == kCtlV) {
         // =====================================================================================
-        // value-side control: V tiles and the value MMAs (chunk dx of block blk -> TMEM slot dx)
+        // value-side control: the value MMAs (chunk c = 3 blk + dx -> TMEM slot c & 1).  One thing to
+        // wait for at a time, so the thread parks in the (bounded) waits.
         // =====================================================================================
         if (lane == 0 && ok) {
             const uint32_t sB0 = smem_u32(smem + L.b_off);
-            bool weights_done = false;
-            int blk = 0, dx = 0;
-            int left = my_tiles - v_issued + 3 * my_blocks;
-            uint32_t idle = 0;
-            while (left > 0) {
-                if (!weights_done) weights_done = mbar_test(bar(kBarWeightsDone), 0);
+            for (int blk = 0; ok && blk < my_blocks; ++blk) {
                 const int eb = blk & 1;
-                const uint32_t tV = mbar_test_u32(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
-                const uint32_t tE = mbar_test_u32(bar(kBarEReady + eb), (blk >> 1) & 1);
-                const int cs = 3 * blk + dx, ds = cs & 1;
-                const uint32_t tD = mbar_test_u32(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1);
-                const int left_before = left;
-                if (tV != 0 && v_issued < my_tiles && (v_issued != SV - 1 || weights_done)) {
-                    issue_v_tile(vq); walk_next(vq, SV); ++v_issued; --left;
-                }
-                if (blk < my_blocks && tE != 0 && tD != 0) {
+                if (!mbar_wait(bar(kBarEReady + eb), (blk >> 1) & 1)) { ok = false; break; }
+                const uint32_t acol = tmem + kColE + 16 * eb;
+#pragma unroll
+                for (int dx = 0; dx < 3; ++dx) {
+                    const int cs = 3 * blk + dx, ds = cs & 1;
+                    if (!mbar_wait(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t sB = sB0 + dx * 12 * 512;
                     const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
                     const uint32_t dcol = tmem + kColD + ds * 112;
-                    const uint32_t acol = tmem + kColE + 16 * eb;
                     umma_bf16_ts(dcol, acol, umma_smem_desc(sB, 128, 512), idesc, 0);
                     umma_bf16_ts(dcol, acol + 8, umma_smem_desc(sB + 256, 128, 512), idesc, 1);
                     umma_commit(bar(kBarDFull + ds));
-                    if (dx == 2) { umma_commit(bar(kBarEFree + eb)); dx = 0; ++blk; }
-                    else ++dx;
-                    --left;
+                    if (dx == 2) umma_commit(bar(kBarEFree + eb));
+                }
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    } else {
+        // =====================================================================================
+        // TMA thread: refills the K/q ring and the V ring as their stages are released
+        // =====================================================================================
+        if (lane == 0 && ok) {
+            bool weights_done = false;
+            int left = my_tiles - v_issued + my_tiles - k_issued;
+            uint32_t idle = 0;
+            while (left > 0) {
+                if (!weights_done) weights_done = mbar_test(bar(kBarWeightsDone), 0);
+                const uint32_t tK = mbar_test_u32(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1);
+                const uint32_t tV = mbar_test_u32(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
+                const int left_before = left;
+                if (tK != 0 && k_issued < my_tiles) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; --left; }
+                // the last V stage held the weights: its first tile waits until every warp is done with them
+                if (tV != 0 && v_issued < my_tiles && (v_issued != SV - 1 || weights_done)) {
+                    issue_v_tile(vq); walk_next(vq, SV); ++v_issued; --left;
                 }
                 if (left != left_before) idle = 0;
-                else if (++idle > (1u << 24)) { ok = false; break; }
+                else {
+                    if (++idle > (1u << 22)) { ok = false; break; }
+                    __nanosleep(200);
+                }
             }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;

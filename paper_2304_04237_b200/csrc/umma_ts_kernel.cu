@@ -429,6 +429,8 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     uint32_t dr[48];
                     const uint32_t ta = tq + colbase;
                     tmem_ld3_16x256b_x4_nowait(ta, ta + 32, ta + 64, dr);
+                    uint32_t sr[4] = {0u, 0u, 0u, 0u};             // sum_s e[p,s] of the two pixels (last chunk)
+                    if (dx == 2) tmem_ld_16x256b_x1_nowait(tq + colbase + 96, sr);
                     uint4 vp[4];
 #pragma unroll
                     for (int r = 0; r < 4; ++r) vp[r] = lds_u4(sV, off0 + (uint32_t)((2 * m + r) * HW2 + dx) * 64u);
@@ -442,6 +444,10 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
                     }
                     tmem_wait_ld48(dr);
+                    if (dx == 2) {
+                        tmem_pass4(sr);
+                        inv[0] = rcp_approx(__uint_as_float(sr[0])); inv[1] = rcp_approx(__uint_as_float(sr[2]));
+                    }
                     float d[48];
 #pragma unroll
                     for (int i = 0; i < 48; ++i) d[i] = __uint_as_float(dr[i]);
@@ -455,11 +461,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                                   vf[dy + 1][2 * j], vf[dy + 1][2 * j + 1]);
                         }
                     }
-                }
-                if (dx == 2) {
-                    float s0[4];
-                    tmem_ld_16x256b_x1(tq + colbase + 96, s0);
-                    inv[0] = rcp_approx(s0[0]); inv[1] = rcp_approx(s0[2]);
                 }
                 tc_fence_before_sync();
                 __syncwarp();

@@ -69,6 +69,29 @@ def ncu_traffic(variant, workload):
     return rec["bytes"] if h == rec["sha256"] else None
 
 
+def other_rooflines(cfg, kernel_ms):
+    """The method's own arithmetic against the two compute ceilings, for context beside the HBM figure:
+    2 C (2 k^4 + 2 k^2) flops per query pixel; fp32 ALU ceiling = SMs x 128 lanes x 2 x max SM clock;
+    bf16 tensor ceiling = the measured cuBLAS figure (burst)."""
+    k2 = cfg["ksize"] ** 2
+    flops = 2.0 * cfg["heads"] * cfg["head_dim"] * (2 * k2 * k2 + 2 * k2) * cfg["B"] * cfg["H"] * cfg["W"]
+    out = {"flops_per_launch": flops}
+    if not kernel_ms or kernel_ms <= 0:
+        return out
+    tf = flops / (kernel_ms * 1e-3) / 1e12
+    out["achieved_tflops"] = tf
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            mp = json.load(f)
+        alu = 148 * 128 * 2 * float(mp["sm_max_mhz"]) * 1e6 / 1e12
+        out.update({"fp32_alu_peak_tflops": alu, "frac_fp32_alu_peak": tf / alu,
+                    "bf16_tensor_peak_tflops": float(mp["bf16_tflops"]),
+                    "frac_bf16_tensor_peak": tf / float(mp["bf16_tflops"])})
+    except Exception:
+        pass
+    return out
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -348,6 +371,7 @@ def main():
                          "traffic": ncu_traffic(variant, args.workload),
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": abytes,
                          "kernel_ms": main_ms, "forward_ms": fwd_ms, "launches_averaged": n_prof},
+            "compute_ceilings": other_rooflines(cfg, main_ms),
             "clocks": clocks, "e2e": e2e,
         }
         if world == 1 and not args.no_cpu_baseline:

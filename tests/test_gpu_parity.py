@@ -286,3 +286,19 @@ def test_wrong_architecture_is_refused_not_emulated():
     with pytest.raises(sa.SlideAttnError) as e:
         sa.slide_attn_create(1, 4, 4, 1, 32, 3, torch.float32, False)
     assert e.value.status == sa.ERR_ARCH
+
+
+def test_auto_random_shapes_against_oracle():
+    """A seeded sweep of small random shapes (odd widths, H or W below the window, more heads than
+    fit one round of CTAs, partial last blocks) through what AUTO runs for bf16 / head_dim 32 /
+    k = 3, element by element against the oracle, each shape twice for bit-identical repeats."""
+    rng = np.random.default_rng(20304)
+    for it in range(48):
+        B, H, W, heads = (int(rng.integers(1, 4)), int(rng.integers(1, 36)), int(rng.integers(1, 140)),
+                          int(rng.integers(1, 8)))
+        x = synth.make_inputs(B, H, W, heads, 32, 3, "bf16", 0.05, 0.2, bool(it & 1), seed=7000 + it)
+        ref = oracle.forward(x["q"], x["k"], x["v"], x["wk"], x["wv"], x["bias"], 3)
+        got = gpu_forward(x, 3, "bf16")
+        again = gpu_forward(x, 3, "bf16")
+        assert np.array_equal(got, again), (B, H, W, heads)
+        assert_close(got, ref, "bf16", f"random shape {(B, H, W, heads)}")

@@ -50,7 +50,7 @@ def algorithmic_bytes(cfg) -> int:
 NCU_TRAFFIC = {
     ("umma_ts", "c2"): {"bytes": 82.24e6,
                         "sources": ("paper_2304_04237_b200/csrc/umma_ts_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
-                        "sha256": "de2983291fc059ba27a0b6e21e7440a0c8ab3f82d5884bf6c85a1fe9a41f909f"},
+                        "sha256": "929fc54088367b41fe45a58c16d15e11ee3947a553ddd656d404b12858846330"},
     ("umma", "c2"): {"bytes": 82.36e6,
                      "sources": ("paper_2304_04237_b200/csrc/umma_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
                      "sha256": "0090172eb4f584d7212bad0870e88367438a5d464ef7a47c3c7544ef734892c1"},

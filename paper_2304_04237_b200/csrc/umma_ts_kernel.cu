@@ -198,7 +198,8 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
     };
 
-    // weights staged in the last V stage; first K tiles and V tiles go out at once
+    // weights are staged in the last V stage; the weights, the first K/q tiles and the first V tiles
+    // are sent for at once
     const unsigned char* w_stage = smem + L.v_off + (size_t)(SV - 1) * L.halo_pad;
     int k_issued = 0, v_issued = 0;
     TileWalk kq = walk_begin(), vq = kq;
@@ -274,7 +275,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     if (warp >= kVWarps && warp < kCtlK) {
         // =====================================================================================
-        // product warps: quadrant q of every block = unit 4 blk + q
+        // product warps: warp (q, pm) takes pixel rows 2pm, 2pm+1 of unit 4 blk + q of every block
         // =====================================================================================
         const int q = (warp - kVWarps) & 3;                        // == warp % 4
         const int pm = (warp - kVWarps) >> 2;                      // pixel-row pair of the unit; softmax of blocks = pm mod 2
@@ -501,10 +502,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (lane == 0) mbar_arrive(bar(kBarVDone));
     } else if (warp == kCtlK || warp == kCtlK2) {
         // =====================================================================================
-        // key-side control: K/q tiles (warp 12) and the key MMAs (18 per block: 9 taps x two K = 16
-        // halves); warp 12 takes the even blocks, warp 14 the odd ones.  Chunks are CLAIMED in order
-        // through one word, so a P-ready barrier is only ever tested for its current or its just
-        // completed phase; the MMAs themselves go out side by side.
+        // key-side control: the key MMAs (18 per block: 9 taps x two K = 16 halves); warp 16 takes
+        // the even blocks, warp 18 the odd ones, in turn.  The tensor pipe executes one small MMA
+        // at a time, so the two threads overlap each other's waits rather than their MMAs.
         // =====================================================================================
         if (lane == 0 && ok) {
             const uint32_t sBk0 = smem_u32(smem + L.bk_off);

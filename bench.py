@@ -92,6 +92,23 @@ def other_rooflines(cfg, kernel_ms):
     return out
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: what a batch sharded over `world` ranks takes (no data-path collective;
+    this all-reduce of one number is the only exchange)."""
+    if world == 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, units_per_rank: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank processes its own full batch, so the job's rate is the sum."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -318,14 +335,10 @@ def main():
     clocks = sampler.stop()
     fwd_ms, main_ms, n_prof = sa.slide_attn_profile_end(ctx)
     assert sa.slide_attn_query_status(ctx) == sa.OK
-    total_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
     ms_per_step = total_ms / args.steps
     npx = cfg["B"] * cfg["H"] * cfg["W"]
-    value = world * npx / (ms_per_step * 1e-3)
+    value = whole_job_value(world, npx, ms_per_step)
 
     # end to end through the host-buffer entry point: pinned host inputs in, pinned result out
     e2e = None
@@ -343,13 +356,9 @@ def main():
             sa.slide_attn_forward_host(ctx, pin["q"], pin["k"], pin["v"], pwk, pwv, pb, pout, stream)
         b.record(stream)
         fence()
-        e2e_ms = a.elapsed_time(b) / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(a.elapsed_time(b) / args.e2e_steps, world, "cuda")
         h2d = 3 * pin["q"].numel() * pin["q"].element_size() + 2 * pwk.numel() * 4 + (0 if pb is None else pb.numel() * 4)
-        e2e = {"value": world * npx / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e = {"value": whole_job_value(world, npx, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(pout.numel() * pout.element_size()),
                "steps": args.e2e_steps}
     sa.slide_attn_destroy(ctx)

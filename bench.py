@@ -53,7 +53,7 @@ NCU_TRAFFIC = {
                         "sha256": "929fc54088367b41fe45a58c16d15e11ee3947a553ddd656d404b12858846330"},
     ("umma", "c2"): {"bytes": 82.36e6,
                      "sources": ("paper_2304_04237_b200/csrc/umma_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
-                     "sha256": "0090172eb4f584d7212bad0870e88367438a5d464ef7a47c3c7544ef734892c1"},
+                     "sha256": "e6187f91a3111cecdd746131ef0e72057c2aa4244a0aab58edba8035ca0a52c9"},
 }
 
 

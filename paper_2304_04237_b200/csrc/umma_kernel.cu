@@ -112,9 +112,6 @@ constexpr int kBarDFull = 22;        // [TMEM slot]  MMA results of a chunk are 
 constexpr int kBarDFree = 26;        // [TMEM slot]  the 4 value warps of the set are done reading the chunk
 constexpr int kBarVDone = 30;        // value warps have finished all TMEM reads
 
-__device__ __forceinline__ float4 lds_f4(const unsigned char* base, uint32_t off) {
-    return *reinterpret_cast<const float4*>(base + off);
-}
 __device__ __forceinline__ uint4 lds_u4(const unsigned char* base, uint32_t off) {
     return *reinterpret_cast<const uint4*>(base + off);
 }

@@ -113,6 +113,9 @@ constexpr int kBarTurn = 35;         // [2]  the other key-control thread has ta
 __device__ __forceinline__ uint4 lds_u4(const unsigned char* base, uint32_t off) {
     return *reinterpret_cast<const uint4*>(base + off);
 }
+// Hand-offs of tensor memory between threads: the side that has read or written TMEM issues
+// tcgen05.wait::ld / ::st (the accesses are then complete) and arrives on an mbarrier; the side that
+// takes over waits on it and issues tcgen05.fence::after_thread_sync before its own tcgen05 work.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
 }
@@ -291,7 +294,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tc_fence_after_sync();
             float Lg[32];
             tmem_ld_32x32b_x32(tq + kColL + 32 * lb, Lg);
-            tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarLFree + lb));
             uint32_t row[16];
@@ -321,7 +323,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tc_fence_after_sync();
             tmem_st_32x32b_x16(tq + kColE + 16 * lb, row);
             tmem_wait_st();
-            tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEReady + lb));
             return true;
@@ -372,7 +373,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         tmem_st_16x256b_x2(tq + ((uint32_t)(16 * pm) << 16) + kColP + 48 * pb + 16 * dy, r);
                     }
                     tmem_wait_st();
-                    tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarPReady + pb));
                 }
@@ -463,7 +463,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         }
                     }
                 }
-                tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
             }

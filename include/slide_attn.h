@@ -124,10 +124,14 @@ slide_attn_status slide_attn_forward(slide_attn_ctx* ctx,
 
 /*
  * The same forward (Eq. 2, Eq. 12, Sec. 4.3) for HOST buffers of the same layouts: copies q, k,
- * v, wk, wv, bias to device staging buffers owned by the context, runs slide_attn_forward,
- * copies `out` back and waits for the stream.  Page-locked host buffers make the copies
- * asynchronous with respect to other streams; pageable ones work too.  The staging buffers are
- * allocated on the first call (cudaMalloc) and reused afterwards.
+ * v, wk, wv, bias to device staging buffers owned by the context, runs the forward, copies `out`
+ * back and waits until all of that is done.  The images of a batch are independent, so the batch
+ * goes through in up to four slices: while one slice is computed on `cuda_stream`, the next one
+ * is copied in and the one before is copied out on two copy streams owned by the context (both
+ * directions of the host link are then busy at once).  The call starts after the work already in
+ * `cuda_stream` and returns with nothing of its own in flight.  Page-locked host buffers are
+ * needed for the copies to overlap; pageable ones work too.  The staging buffers, the copy
+ * streams and their events are created on the first call and reused afterwards.
  */
 slide_attn_status slide_attn_forward_host(slide_attn_ctx* ctx,
                                           const void* q, const void* k, const void* v,

@@ -259,10 +259,12 @@ def test_forward_argument_errors():
         sa.slide_attn_destroy(ctx)
 
 
+@pytest.mark.parametrize("B,H,W", [(2, 11, 13), (1, 9, 20), (7, 56, 56)])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_host_buffer_entry_point(dtype):
-    """slide_attn_forward_host (host buffers in and out) gives the device path's result."""
-    B, H, W, heads, d, k = 2, 11, 13, 2, 32, 3
+def test_host_buffer_entry_point(dtype, B, H, W):
+    """slide_attn_forward_host (host buffers in and out) gives the device path's result; the batch
+    sizes cover one slice, two small slices and four uneven slices of its copy / compute pipeline."""
+    heads, d, k = 2, 32, 3
     x = synth.make_inputs(B, H, W, heads, d, k, dtype, 0.05, 0.1, True, seed=123)
     td = TORCH_DTYPE[dtype]
     host = {n: torch.from_numpy(x[n]).to(td).pin_memory() for n in ("q", "k", "v")}

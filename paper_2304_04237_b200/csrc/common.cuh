@@ -35,6 +35,13 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(f
 cudaError_t launch_direct(const Problem& p, cudaStream_t stream);
 bool direct_supports(int head_dim, int ksize);
 
+// STRIP variant: generic fp32 path with transposed weights (strip_workspace_bytes, written by the
+// prep launch of every forward) and four pixels per warp.
+bool strip_supports(int head_dim, int ksize);
+size_t strip_workspace_bytes(int heads, int head_dim, int ksize);
+cudaError_t launch_strip_prep(const Problem& p, void* workspace, cudaStream_t stream);
+cudaError_t launch_strip_main(const Problem& p, const void* workspace, cudaStream_t stream);
+
 // MMA variant.  `workspace` holds the re-laid-out weights (mma_workspace_bytes), written by the
 // prep launch and read by the main launch on the same stream.  mma_setup must have succeeded once
 // on the device before the first main launch.

@@ -15,6 +15,7 @@ struct slide_attn_ctx {
     int* d_status;                   // device status word (0 = ok)
     void* workspace;                 // re-laid-out weights for the variants that need them
     size_t workspace_bytes;
+    void* strip_ws;                  // transposed weights of the STRIP variant
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
     size_t stage_bytes;
@@ -39,6 +40,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
     switch (v) {
         case SLIDE_ATTN_VARIANT_DIRECT: return direct_supports(c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_STRIP: return c->strip_ws && strip_supports(c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_MMA: return c->workspace && mma_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_MMA_WS: return mma_ws_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA: return umma_supports(c->dtype, c->head_dim, c->ksize);
@@ -49,7 +51,8 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
 
 slide_attn_variant pick_variant(const slide_attn_ctx* c) {
     const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA_TS, SLIDE_ATTN_VARIANT_UMMA, SLIDE_ATTN_VARIANT_MMA_WS,
-                                        SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_DIRECT};
+                                        SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_STRIP,
+                                        SLIDE_ATTN_VARIANT_DIRECT};
     for (slide_attn_variant v : order)
         if (variant_supported(c, v)) return v;
     return SLIDE_ATTN_VARIANT_DIRECT;
@@ -81,6 +84,11 @@ slide_attn_status launch_problem(slide_attn_ctx* c, const Problem& p, cudaStream
         case SLIDE_ATTN_VARIANT_DIRECT:
             if (ev) cudaEventRecord(ev[1], stream);
             err = launch_direct(p, stream);
+            break;
+        case SLIDE_ATTN_VARIANT_STRIP:
+            err = launch_strip_prep(p, c->strip_ws, stream);
+            if (ev) cudaEventRecord(ev[1], stream);
+            if (err == cudaSuccess) err = launch_strip_main(p, c->strip_ws, stream);
             break;
         case SLIDE_ATTN_VARIANT_MMA:
             err = launch_mma_prep(p, c->workspace, stream);
@@ -163,6 +171,13 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
             slide_attn_destroy(c);
             return SLIDE_ATTN_ERR_ALLOC;
         }
+    }
+    if (strip_supports(head_dim, ksize) &&
+        cudaMalloc(&c->strip_ws, strip_workspace_bytes(heads, head_dim, ksize)) != cudaSuccess) {
+        cudaGetLastError();
+        c->strip_ws = nullptr;
+        slide_attn_destroy(c);
+        return SLIDE_ATTN_ERR_ALLOC;
     }
     c->variant = pick_variant(c);
     *ctx = c;
@@ -275,7 +290,7 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant v
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (variant == SLIDE_ATTN_VARIANT_AUTO) { c->variant = pick_variant(c); return SLIDE_ATTN_OK; }
-    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_UMMA_TS)
+    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_STRIP)
         return SLIDE_ATTN_ERR_INVALID_ARG;
     if (!variant_supported(c, variant)) return SLIDE_ATTN_ERR_UNSUPPORTED;
     c->variant = variant;
@@ -295,6 +310,7 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
     switch (c->variant) {
         case SLIDE_ATTN_VARIANT_DIRECT: *n = 1; break;
         case SLIDE_ATTN_VARIANT_MMA: *n = 2; break;      // weight re-layout + fused kernel
+        case SLIDE_ATTN_VARIANT_STRIP: *n = 2; break;    // weight transpose + fused kernel
         case SLIDE_ATTN_VARIANT_MMA_WS: *n = 1; break;
         case SLIDE_ATTN_VARIANT_UMMA: *n = 1; break;
         case SLIDE_ATTN_VARIANT_UMMA_TS: *n = 1; break;
@@ -368,6 +384,7 @@ slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
     bool ok = true;
     if (c->d_status) ok &= cudaFree(c->d_status) == cudaSuccess;
     if (c->workspace) ok &= cudaFree(c->workspace) == cudaSuccess;
+    if (c->strip_ws) ok &= cudaFree(c->strip_ws) == cudaSuccess;
     if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
     if (c->host_pipe) {
         ok &= cudaStreamDestroy(c->copy_in) == cudaSuccess;

@@ -15,7 +15,7 @@ from util import TORCH_DTYPE, VARIANTS, assert_close, gpu_forward, to_device
 
 pytestmark = pytest.mark.gpu
 
-ALL_VARIANTS = ["auto", "direct", "mma", "mma_ws", "umma", "umma_ts"]
+ALL_VARIANTS = ["auto", "direct", "strip", "mma", "mma_ws", "umma", "umma_ts"]
 
 
 def ref_forward(x, k):

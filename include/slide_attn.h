@@ -43,7 +43,9 @@
  *
  * Threading: one context must not be used from two host threads at once, and two forwards on
  * the same context must be ordered on the device (same stream, or events), because they share
- * the context's workspace.  Distinct contexts are independent.
+ * the context's workspace.  Distinct contexts are independent.  A context belongs to the device
+ * that was current when it was created: forward, forward_host and query_status return
+ * SLIDE_ATTN_ERR_INVALID_ARG, before launching anything, when another device is current.
  */
 #ifndef SLIDE_ATTN_H_
 #define SLIDE_ATTN_H_
@@ -169,17 +171,21 @@ slide_attn_status slide_attn_query_status(slide_attn_ctx* ctx, void* cuda_stream
  * device synchronisation of cudaMalloc / cudaFree.  slide_attn_create allocates, so such callers
  * cannot use a context.  Here the scratch memory of the tensor-core variant (re-laid-out weights,
  * status word) is a fixed array inside the library's device image instead; every GPU that loads
- * the library holds it (288.25 KiB) until the process exits.  This call performs no cudaMalloc,
- * cudaFree or other allocating call.
+ * the library holds it (288.25 KiB) from the moment the driver loads the library's device code on
+ * that GPU until the process exits.  This call itself performs no cudaMalloc, cudaFree or other
+ * allocating call.
  *
  * Arguments: tensors as for slide_attn_forward (DEVICE pointers, same layouts, 16-byte aligned,
  * bias may be NULL), followed by the shape the context would have carried.
  * Limits: dtype SLIDE_ATTN_BF16, head_dim 32, ksize 3 (else SLIDE_ATTN_ERR_UNSUPPORTED);
  * heads <= 16 (else SLIDE_ATTN_ERR_TOO_LARGE -- the fixed scratch has room for 16 heads).
  *
- * First call on a device: resolves the scratch's device address and configures the kernel
- * (no allocation, but driver calls that are not legal during stream capture) -- make the first
- * call on each device outside of any stream capture, with that device current.
+ * First call on a device: resolves the scratch's device address and configures the kernel.  With
+ * CUDA's lazy module loading this is also when the driver may load the library's device code,
+ * which takes device memory inside the driver (the scratch array included) and is not legal during
+ * stream capture.  So make the first call on each device during start-up, with that device current,
+ * outside of any stream capture and before an allocator is frozen.  Later calls on that device make
+ * no allocating call of any kind.
  *
  * Sharing: every call on a device uses the same scratch, and the scratch keeps the previous call's
  * contents.  Each call rewrites all of it that it reads and clears the status word first, so

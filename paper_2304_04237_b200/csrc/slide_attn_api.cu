@@ -37,6 +37,14 @@ size_t elem_size(slide_attn_dtype t) { return t == SLIDE_ATTN_BF16 ? 2 : 4; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The context's workspace, status word and streams belong to the device it was created on; a launch
+// with another device current would hand that device foreign pointers.
+bool on_ctx_device(const slide_attn_ctx* c) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+    return dev == c->device;
+}
+
 bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
     switch (v) {
         case SLIDE_ATTN_VARIANT_DIRECT: return direct_supports(c->head_dim, c->ksize);
@@ -191,6 +199,7 @@ slide_attn_status slide_attn_forward(slide_attn_ctx* c, const void* q, const voi
     if (!c || !q || !k || !v || !wk || !wv || !out) return SLIDE_ATTN_ERR_INVALID_ARG;
     if ((c->has_bias != 0) != (bias != nullptr)) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(wk) ||
         !aligned16(wv) || (bias && !aligned16(bias)))
         return SLIDE_ATTN_ERR_ALIGNMENT;
@@ -208,6 +217,7 @@ slide_attn_status slide_attn_forward_host(slide_attn_ctx* c, const void* q, cons
 {
     if (!c || !q || !k || !v || !wk || !wv || !out) return SLIDE_ATTN_ERR_INVALID_ARG;
     if ((c->has_bias != 0) != (bias != nullptr)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     const size_t C = (size_t)c->heads * c->head_dim, k2 = (size_t)c->ksize * c->ksize;
@@ -366,7 +376,7 @@ slide_attn_status slide_attn_profile_end(slide_attn_ctx* c, double* forward_ms, 
 
 slide_attn_status slide_attn_query_status(slide_attn_ctx* c, void* cuda_stream)
 {
-    if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!c || !on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int word = 0;
     if (cudaMemcpyAsync(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||

@@ -68,9 +68,7 @@ struct UmmaParams {
     __nv_bfloat16* out;
     int* status;
     int B, H, W, heads;
-    int TW;
     int tiles_x, tiles_y;
-    int stages;
     float scale_log2e;
 };
 
@@ -78,8 +76,8 @@ struct Smem {
     uint32_t halo_pad, kstage_bytes, v_off, b_off, bk_off, tmem_off, bar_off, total;
 };
 
-__host__ __device__ inline Smem smem_layout(int TW, int vstages) {
-    Smem s;
+__host__ __device__ constexpr Smem smem_layout(int TW, int vstages) {
+    Smem s{};
     s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 1023u) & ~1023u;
     const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
     if (s.halo_pad < wbytes) s.halo_pad = wbytes;
@@ -91,6 +89,16 @@ __host__ __device__ inline Smem smem_layout(int TW, int vstages) {
     s.bar_off = s.tmem_off + 16;
     s.total = s.bar_off + 40 * 8 + 1024;
     return s;
+}
+
+constexpr size_t kMaxSmem = 227 * 1024;
+
+// V stages that fit beside everything else for a tile width (the kernel is instantiated per width,
+// so that every shared-memory offset and stride is a compile-time constant)
+__host__ __device__ constexpr int v_stages_for(int TW) {
+    for (int st = kMaxVStages; st >= 2; --st)
+        if (smem_layout(TW, st).total <= kMaxSmem) return st;
+    return 0;
 }
 
 constexpr int kBarKFull = 0;         // [2]
@@ -120,21 +128,23 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
 }
 
+template <int TW>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
              const __grid_constant__ CUtensorMap map_v, const UmmaParams P)
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    const Smem L = smem_layout(P.TW, P.stages);
+    constexpr int SV = v_stages_for(TW);
+    constexpr Smem L = smem_layout(TW, SV);
     const uint32_t bar0 = smem_u32(smem + L.bar_off);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the warp index through a shuffle: the compiler then knows it is the same in every lane
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int g = lane >> 2, tig = lane & 3;
-    const int SV = P.stages;
-    const int U = P.TW >> 3;
-    const int HW2 = P.TW + 2;
+    constexpr int U = TW >> 3;
+    constexpr int HW2 = TW + 2;
 
     const int h = blockIdx.x % P.heads;
     const int rank = blockIdx.x / P.heads;
@@ -190,15 +200,15 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     auto issue_k_tile = [&](const TileWalk& w) {
         const uint32_t base = smem_u32(smem + (size_t)w.stage * L.kstage_bytes);
         const uint32_t fb = bar(kBarKFull + w.stage);
-        mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64 + 4 * P.TW * 64));
-        tma_load_4d(base, &map_k, fb, h * kHeadDim, w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
-        tma_load_4d(base + L.halo_pad, &map_q, fb, h * kHeadDim, w.tx * P.TW, w.ty * 4, w.b);
+        mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64 + 4 * TW * 64));
+        tma_load_4d(base, &map_k, fb, h * kHeadDim, w.tx * TW - 1, w.ty * 4 - 1, w.b);
+        tma_load_4d(base + L.halo_pad, &map_q, fb, h * kHeadDim, w.tx * TW, w.ty * 4, w.b);
     };
     auto issue_v_tile = [&](const TileWalk& w) {
         const uint32_t fb = bar(kBarVFull + w.stage);
         mbar_expect_tx(fb, (uint32_t)(6 * HW2 * 64));
         tma_load_4d(smem_u32(smem + L.v_off + (size_t)w.stage * L.halo_pad), &map_v, fb, h * kHeadDim,
-                    w.tx * P.TW - 1, w.ty * 4 - 1, w.b);
+                    w.tx * TW - 1, w.ty * 4 - 1, w.b);
     };
 
     // weights are staged in the last V stage; the weights, the first K/q tiles and the first V tiles
@@ -211,9 +221,14 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
         bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
     }
-    if (my_tiles > 0 && warp == kCtlT && lane == 0) {
-        while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
-        while (v_issued < my_tiles && v_issued < SV - 1) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
+    if (my_tiles > 0 && warp == kCtlT) {
+        // the same lane is elected here and in the refill loop below (the election is deterministic for
+        // a given member mask), so the ring positions it advances here are the ones it continues from
+        uint32_t leader;
+        if (elect_one(leader)) {
+            while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
+            while (v_issued < my_tiles && v_issued < SV - 1) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
+        }
     }
     __syncwarp();
 
@@ -350,7 +365,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 uint32_t qf[2][4];                                 // pixel rows 2pm, 2pm+1 of column ux + g
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
-                    const uint4 v = lds_u4(sQ, (uint32_t)((2 * pm + i) * P.TW + ux + g) * 64u + tig * 16u);
+                    const uint4 v = lds_u4(sQ, (uint32_t)((2 * pm + i) * TW + ux + g) * 64u + tig * 16u);
                     qf[i][0] = v.x; qf[i][1] = v.y; qf[i][2] = v.z; qf[i][3] = v.w;
                 }
                 const uint32_t off0 = (uint32_t)(ux + g) * 64u + tig * 16u;
@@ -469,7 +484,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             if (!ok) break;
 
             {
-                const int x = tx * P.TW + ux + g, y0 = ty * 4 + 2 * m;
+                const int x = tx * TW + ux + g, y0 = ty * 4 + 2 * m;
                 __nv_bfloat16* op = P.out + ((size_t)(b * P.H + y0) * P.W + x) * C + h * kHeadDim + tig * 8;
                 const size_t row_stride = (size_t)P.W * C;
 #pragma unroll
@@ -505,7 +520,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // the even blocks, warp 18 the odd ones, in turn.  The tensor pipe executes one small MMA
         // at a time, so the two threads overlap each other's waits rather than their MMAs.
         // =====================================================================================
-        if (lane == 0 && ok) {
+        uint32_t leader;
+        const bool elected = elect_one(leader);
+        if (elected && ok) {
             const uint32_t sBk0 = smem_u32(smem + L.bk_off);
             // This thread has one thing to wait for at a time, so it parks in the waits (bounded).
             // The two threads take the blocks in turn: a thread starts block b only when the other
@@ -539,7 +556,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
             }
         }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
         if (warp == kCtlK) {
             if (my_tiles > 0 && !warp_wait(bar(kBarVDone), 0)) ok = false;
             tc_fence_after_sync();
@@ -551,7 +568,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // value-side control: the value MMAs (chunk c = 3 blk + dx -> TMEM slot c & 1).  One thing to
         // wait for at a time, so the thread parks in the (bounded) waits.
         // =====================================================================================
-        if (lane == 0 && ok) {
+        uint32_t leader;
+        const bool elected = elect_one(leader);
+        if (elected && ok) {
             const uint32_t sB0 = smem_u32(smem + L.b_off);
             for (int blk = 0; ok && blk < my_blocks; ++blk) {
                 const int eb = blk & 1;
@@ -572,12 +591,14 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
             }
         }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
     } else {
         // =====================================================================================
         // TMA thread: refills the K/q ring and the V ring as their stages are released
         // =====================================================================================
-        if (lane == 0 && ok) {
+        uint32_t leader;
+        const bool elected = elect_one(leader);
+        if (elected && ok) {
             bool weights_done = false;
             int left = my_tiles - v_issued + my_tiles - k_issued;
             uint32_t idle = 0;
@@ -598,7 +619,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
             }
         }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
     }
     if (!ok && my_tiles > 0 && lane == 0) atomicExch(P.status, 1);
 }
@@ -633,17 +654,40 @@ bool make_map(CUtensorMap* map, const void* base, int B, int H, int W, int C, in
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t kMaxSmem = 227 * 1024;
-
 }  // namespace
 
 bool umma_ts_supports(slide_attn_dtype dtype, int head_dim, int ksize) {
     return dtype == SLIDE_ATTN_BF16 && head_dim == kHeadDim && ksize == 3;
 }
 
+namespace {
+
+template <int TW>
+cudaError_t setup_one() {
+    return cudaFuncSetAttribute(umma_ts_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+}
+
+template <int TW>
+cudaError_t launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& P,
+                       int grid, cudaStream_t stream) {
+    static_assert(v_stages_for(TW) >= 2, "tile width does not fit shared memory");
+    umma_ts_kernel<TW><<<grid, kThreads, smem_layout(TW, v_stages_for(TW)).total, stream>>>(mq, mk, mv, P);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
 cudaError_t umma_ts_setup() {
     if (!encode_fn()) return cudaErrorNotSupported;
-    return cudaFuncSetAttribute(umma_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+    cudaError_t e = setup_one<8>();
+    if (e == cudaSuccess) e = setup_one<16>();
+    if (e == cudaSuccess) e = setup_one<24>();
+    if (e == cudaSuccess) e = setup_one<32>();
+    if (e == cudaSuccess) e = setup_one<40>();
+    if (e == cudaSuccess) e = setup_one<48>();
+    if (e == cudaSuccess) e = setup_one<56>();
+    if (e == cudaSuccess) e = setup_one<64>();
+    return e;
 }
 
 cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStream_t stream) {
@@ -654,15 +698,9 @@ cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStr
     P.out = static_cast<__nv_bfloat16*>(p.out);
     P.status = d_status;
     P.B = p.B; P.H = p.H; P.W = p.W; P.heads = p.heads;
-    P.TW = TW;
     P.tiles_x = (p.W + TW - 1) / TW;
     P.tiles_y = (p.H + 3) / 4;
-    P.stages = 2;
-    for (int st = kMaxVStages; st >= 2; --st)
-        if (smem_layout(TW, st).total <= kMaxSmem) { P.stages = st; break; }
     P.scale_log2e = kLog2e / sqrtf((float)kHeadDim);
-    const Smem L = smem_layout(TW, P.stages);
-    if (L.total > kMaxSmem) return cudaErrorInvalidConfiguration;
 
     const int C = p.heads * kHeadDim;
     CUtensorMap map_q, map_k, map_v;
@@ -676,8 +714,17 @@ cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStr
     int grid = num_sms;
     if (grid < p.heads) grid = p.heads;
     if ((long long)grid > tiles) grid = (int)tiles;
-    umma_ts_kernel<<<grid, kThreads, L.total, stream>>>(map_q, map_k, map_v, P);
-    return cudaGetLastError();
+    switch (TW) {
+        case 8: return launch_one<8>(map_q, map_k, map_v, P, grid, stream);
+        case 16: return launch_one<16>(map_q, map_k, map_v, P, grid, stream);
+        case 24: return launch_one<24>(map_q, map_k, map_v, P, grid, stream);
+        case 32: return launch_one<32>(map_q, map_k, map_v, P, grid, stream);
+        case 40: return launch_one<40>(map_q, map_k, map_v, P, grid, stream);
+        case 48: return launch_one<48>(map_q, map_k, map_v, P, grid, stream);
+        case 56: return launch_one<56>(map_q, map_k, map_v, P, grid, stream);
+        case 64: return launch_one<64>(map_q, map_k, map_v, P, grid, stream);
+        default: return cudaErrorInvalidConfiguration;
+    }
 }
 
 }  // namespace slide_attn

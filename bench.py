@@ -257,7 +257,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
-    ap.add_argument("--variant", default="auto", choices=["auto", "direct", "mma", "mma_ws", "umma", "umma_ts", "strip"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "direct", "mma", "mma_ws", "umma", "umma_ts", "strip", "umma_sp"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -304,8 +304,8 @@ def main():
     ctx = sa.slide_attn_create(cfg["B"], cfg["H"], cfg["W"], cfg["heads"], cfg["head_dim"],
                                cfg["ksize"], td, cfg["has_bias"])
     if args.variant != "auto":
-        sa.slide_attn_set_variant(ctx, {"direct": 1, "mma": 2, "mma_ws": 3, "umma": 4, "umma_ts": 5, "strip": 6}[args.variant])
-    variant = {1: "direct", 2: "mma", 3: "mma_ws", 4: "umma", 5: "umma_ts", 6: "strip"}[sa.slide_attn_get_variant(ctx)]
+        sa.slide_attn_set_variant(ctx, {"direct": 1, "mma": 2, "mma_ws": 3, "umma": 4, "umma_ts": 5, "strip": 6, "umma_sp": 7}[args.variant])
+    variant = {1: "direct", 2: "mma", 3: "mma_ws", 4: "umma", 5: "umma_ts", 6: "strip", 7: "umma_sp"}[sa.slide_attn_get_variant(ctx)]
     launches = sa.slide_attn_launches_per_forward(ctx)
     stream = torch.cuda.current_stream()
 

@@ -90,10 +90,14 @@ typedef enum {
     SLIDE_ATTN_VARIANT_UMMA_TS = 5,   /* both contractions on tcgen05.mma with their A operands (the
                                          q.k products, the softmax weights) held in tensor memory;
                                          bf16, head_dim 32, ksize 3                                     */
-    SLIDE_ATTN_VARIANT_STRIP   = 6    /* DIRECT's arithmetic with transposed weights (one coalesced load
+    SLIDE_ATTN_VARIANT_STRIP   = 6,   /* DIRECT's arithmetic with transposed weights (one coalesced load
                                          per weight) and 4-8 pixels per warp; fp32 FMA; ksize <= 9,
                                          any head_dim, fp32 or bf16: what AUTO runs where the tensor-core
                                          variants do not apply                                          */
+    SLIDE_ATTN_VARIANT_UMMA_SP = 7    /* UMMA_TS's arithmetic as one team of eight warps running a
+                                         software pipeline over the pixel blocks (products, softmax and
+                                         value phase of three consecutive blocks per iteration), tensor
+                                         memory single-buffered; bf16, head_dim 32, ksize 3             */
 } slide_attn_variant;
 
 /*

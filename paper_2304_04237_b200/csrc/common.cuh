@@ -1,6 +1,7 @@
 // Shared declarations of the slide-attention library: problem description, element access,
 // and the launchers each kernel file exports to the API layer.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -30,6 +31,12 @@ template <> __device__ __forceinline__ float from_float<float>(float x) { return
 template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float x) {
     return __float2bfloat16_rn(x);
 }
+
+// TMA tensor map of a [B][H][W][C] tensor (bf16: elem_bytes 2, fp32: 4) seen as 4-D (C, W, H, B) with
+// a box of box_c channels x box_w columns x box_h rows; out-of-map elements read as zero.
+bool tensor_map_available();
+bool make_tile_map(CUtensorMap* map, const void* base, int elem_bytes, int B, int H, int W, int C,
+                   int box_c, int box_w, int box_h);
 
 // Launchers.  Each returns cudaGetLastError() of its launch(es).
 cudaError_t launch_direct(const Problem& p, cudaStream_t stream);
@@ -67,5 +74,12 @@ cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream
 bool umma_ts_supports(slide_attn_dtype dtype, int head_dim, int ksize);
 cudaError_t umma_ts_setup();
 cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
+
+// UMMA_SP variant: the tcgen05 arithmetic of UMMA_TS in ONE software-pipelined team of eight warps
+// (every warp forms q.k products, takes its turn at the softmax and applies the value weights), so
+// tensor memory is single-buffered and a block costs four barrier hand-offs instead of twenty.
+bool umma_sp_supports(slide_attn_dtype dtype, int head_dim, int ksize);
+cudaError_t umma_sp_setup();
+cudaError_t launch_umma_sp(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
 
 }  // namespace slide_attn

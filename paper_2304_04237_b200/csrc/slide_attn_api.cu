@@ -53,6 +53,7 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
         case SLIDE_ATTN_VARIANT_MMA_WS: return mma_ws_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA: return umma_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA_TS: return umma_ts_supports(c->dtype, c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_UMMA_SP: return umma_sp_supports(c->dtype, c->head_dim, c->ksize);
         default: return false;
     }
 }
@@ -115,6 +116,10 @@ slide_attn_status launch_problem(slide_attn_ctx* c, const Problem& p, cudaStream
             if (ev) cudaEventRecord(ev[1], stream);
             err = launch_umma_ts(p, c->d_status, c->num_sms, stream);
             break;
+        case SLIDE_ATTN_VARIANT_UMMA_SP:
+            if (ev) cudaEventRecord(ev[1], stream);
+            err = launch_umma_sp(p, c->d_status, c->num_sms, stream);
+            break;
         default: return SLIDE_ATTN_ERR_UNSUPPORTED;
     }
     if (ev) {
@@ -167,7 +172,7 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
     }
     if (mma_supports(dtype, head_dim, ksize)) {
         if (mma_setup() != cudaSuccess || mma_ws_setup() != cudaSuccess || umma_setup() != cudaSuccess ||
-            umma_ts_setup() != cudaSuccess) {
+            umma_ts_setup() != cudaSuccess || umma_sp_setup() != cudaSuccess) {
             cudaGetLastError();
             slide_attn_destroy(c);
             return SLIDE_ATTN_ERR_CUDA;
@@ -300,7 +305,7 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant v
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (variant == SLIDE_ATTN_VARIANT_AUTO) { c->variant = pick_variant(c); return SLIDE_ATTN_OK; }
-    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_STRIP)
+    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_UMMA_SP)
         return SLIDE_ATTN_ERR_INVALID_ARG;
     if (!variant_supported(c, variant)) return SLIDE_ATTN_ERR_UNSUPPORTED;
     c->variant = variant;
@@ -324,6 +329,7 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
         case SLIDE_ATTN_VARIANT_MMA_WS: *n = 1; break;
         case SLIDE_ATTN_VARIANT_UMMA: *n = 1; break;
         case SLIDE_ATTN_VARIANT_UMMA_TS: *n = 1; break;
+        case SLIDE_ATTN_VARIANT_UMMA_SP: *n = 1; break;
         default: *n = 1; break;
     }
     return SLIDE_ATTN_OK;

@@ -70,10 +70,13 @@ bool umma_supports(slide_attn_dtype dtype, int head_dim, int ksize);
 cudaError_t umma_setup();
 cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
 
-// UMMA_TS variant: both contractions on tcgen05 with their A operands in tensor memory.
+// UMMA_TS variant: both contractions on tcgen05 with their A operands in tensor memory.  A prep launch
+// writes the bf16 B images of every head (umma_ts_workspace_bytes) that the main launch's CTAs copy in.
 bool umma_ts_supports(slide_attn_dtype dtype, int head_dim, int ksize);
 cudaError_t umma_ts_setup();
-cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
+size_t umma_ts_workspace_bytes(int heads);
+cudaError_t launch_umma_ts_prep(const Problem& p, void* workspace, cudaStream_t stream);
+cudaError_t launch_umma_ts(const Problem& p, const void* workspace, int* d_status, int num_sms, cudaStream_t stream);
 
 // UMMA_SP variant: the tcgen05 arithmetic of UMMA_TS in ONE software-pipelined team of eight warps
 // (every warp forms q.k products, takes its turn at the softmax and applies the value weights), so

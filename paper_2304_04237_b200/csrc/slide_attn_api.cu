@@ -16,6 +16,7 @@ struct slide_attn_ctx {
     void* workspace;                 // re-laid-out weights for the variants that need them
     size_t workspace_bytes;
     void* strip_ws;                  // transposed weights of the STRIP variant
+    void* umma_ws;                   // bf16 B images of the UMMA_TS variant
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
     size_t stage_bytes;
@@ -52,7 +53,7 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
         case SLIDE_ATTN_VARIANT_MMA: return c->workspace && mma_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_MMA_WS: return mma_ws_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA: return umma_supports(c->dtype, c->head_dim, c->ksize);
-        case SLIDE_ATTN_VARIANT_UMMA_TS: return umma_ts_supports(c->dtype, c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_UMMA_TS: return c->umma_ws && umma_ts_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA_SP: return umma_sp_supports(c->dtype, c->head_dim, c->ksize);
         default: return false;
     }
@@ -113,8 +114,9 @@ slide_attn_status launch_problem(slide_attn_ctx* c, const Problem& p, cudaStream
             err = launch_umma(p, c->d_status, c->num_sms, stream);
             break;
         case SLIDE_ATTN_VARIANT_UMMA_TS:
+            err = launch_umma_ts_prep(p, c->umma_ws, stream);
             if (ev) cudaEventRecord(ev[1], stream);
-            err = launch_umma_ts(p, c->d_status, c->num_sms, stream);
+            if (err == cudaSuccess) err = launch_umma_ts(p, c->umma_ws, c->d_status, c->num_sms, stream);
             break;
         case SLIDE_ATTN_VARIANT_UMMA_SP:
             if (ev) cudaEventRecord(ev[1], stream);
@@ -181,6 +183,12 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
         if (cudaMalloc(&c->workspace, c->workspace_bytes) != cudaSuccess) {
             cudaGetLastError();
             c->workspace = nullptr;
+            slide_attn_destroy(c);
+            return SLIDE_ATTN_ERR_ALLOC;
+        }
+        if (cudaMalloc(&c->umma_ws, umma_ts_workspace_bytes(heads)) != cudaSuccess) {
+            cudaGetLastError();
+            c->umma_ws = nullptr;
             slide_attn_destroy(c);
             return SLIDE_ATTN_ERR_ALLOC;
         }
@@ -328,7 +336,7 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
         case SLIDE_ATTN_VARIANT_STRIP: *n = 2; break;    // weight transpose + fused kernel
         case SLIDE_ATTN_VARIANT_MMA_WS: *n = 1; break;
         case SLIDE_ATTN_VARIANT_UMMA: *n = 1; break;
-        case SLIDE_ATTN_VARIANT_UMMA_TS: *n = 1; break;
+        case SLIDE_ATTN_VARIANT_UMMA_TS: *n = 2; break;  // B-image prep + fused kernel
         case SLIDE_ATTN_VARIANT_UMMA_SP: *n = 1; break;
         default: *n = 1; break;
     }
@@ -401,6 +409,7 @@ slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
     if (c->d_status) ok &= cudaFree(c->d_status) == cudaSuccess;
     if (c->workspace) ok &= cudaFree(c->workspace) == cudaSuccess;
     if (c->strip_ws) ok &= cudaFree(c->strip_ws) == cudaSuccess;
+    if (c->umma_ws) ok &= cudaFree(c->umma_ws) == cudaSuccess;
     if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
     if (c->host_pipe) {
         ok &= cudaStreamDestroy(c->copy_in) == cudaSuccess;

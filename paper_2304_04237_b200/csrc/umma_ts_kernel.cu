@@ -49,7 +49,7 @@ constexpr int kMaxVStages = 4;
 constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
 constexpr int kBBytes = kBCols * 64;
 constexpr int kBkBytes = 36 * 512;                      // key-side B: 288 K x 32 N bf16
-constexpr int kWeightBytes = kHeadDim * 81 * 4;
+constexpr int kImgBytes = kBBytes + kBkBytes;           // both B images of one head, as the prep kernel leaves them
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kTmemCols = 512;
 // tensor-memory columns
@@ -62,8 +62,7 @@ constexpr uint32_t kIdesc112 = umma_idesc_bf16(128, 112);
 constexpr uint32_t kIdesc32 = umma_idesc_bf16(128, 32);
 
 struct UmmaParams {
-    const float* wk;
-    const float* wv;
+    const unsigned char* bimg;       // per head: value-side B image (kBBytes) then key-side B image (kBkBytes)
     const float* bias;
     __nv_bfloat16* out;
     int* status;
@@ -79,8 +78,6 @@ struct Smem {
 __host__ __device__ constexpr Smem smem_layout(int TW, int vstages) {
     Smem s{};
     s.halo_pad = ((uint32_t)(6 * (TW + 2) * 64) + 1023u) & ~1023u;
-    const uint32_t wbytes = ((uint32_t)(2 * kWeightBytes) + 1023u) & ~1023u;
-    if (s.halo_pad < wbytes) s.halo_pad = wbytes;
     s.kstage_bytes = s.halo_pad + (((uint32_t)(4 * TW * 64) + 1023u) & ~1023u);
     s.v_off = kKStages * s.kstage_bytes;
     s.b_off = s.v_off + vstages * s.halo_pad;
@@ -105,8 +102,7 @@ constexpr int kBarKFull = 0;         // [2]
 constexpr int kBarKEmpty = 2;        // [2]  count 8 (product warps)
 constexpr int kBarVFull = 4;         // [4]
 constexpr int kBarVEmpty = 8;        // [4]  count 8
-constexpr int kBarWeights = 12;
-constexpr int kBarWeightsDone = 13;  // count 20 (every warp)
+constexpr int kBarWeights = 12;      // both B images have landed (one bulk copy)
 constexpr int kBarPReady = 14;       // [4]  count 8: P chunk stored by the eight product warps
 constexpr int kBarPFree = 18;        // [4]  key MMAs reading the chunk are complete
 constexpr int kBarLFull = 22;        // [2]  logits of a block complete
@@ -126,6 +122,72 @@ __device__ __forceinline__ uint4 lds_u4(const unsigned char* base, uint32_t off)
 // takes over waits on it and issues tcgen05.fence::after_thread_sync before its own tcgen05 work.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Prep kernel: the two B images of every head, in the shared-memory layout the MMAs read
+// (K-major core matrices of 8 rows x 16 bytes, no swizzle), written to the context workspace once per
+// forward.  Block (h, part) builds a share of head h's items.
+//   value side  [304 columns][32 K] bf16: column n = (tap-column-major tap, channel); K rows
+//               0..7 D_v[c][s][t], 8..15 and 16..23 the one-hot [s = t], 24 D_v[c][8][t], 25, 26 [t = 8]
+//               (the A' row is e_hi | e_hi | e_lo | e8_hi e8_hi e8_lo); columns 288.. sum the A' row
+//   key side    [288 K][32 N] bf16: K = 32 tap + kappa (kappa -> channel as tcgen05.st lays P out),
+//               N 0..8 D_k[c][n][t], 9..17 the one-hot [n - 9 = t]
+__global__ void __launch_bounds__(256)
+umma_ts_prep_kernel(const float* __restrict__ wk, const float* __restrict__ wv, unsigned char* __restrict__ img)
+{
+    grid_launch_dependents();        // the main kernel may start its own prologue now
+    const int h = blockIdx.x;
+    const float* wks = wk + (size_t)h * kHeadDim * 81;
+    const float* wvs = wv + (size_t)h * kHeadDim * 81;
+    unsigned char* sB = img + (size_t)h * kImgBytes;
+    unsigned char* sBk = sB + kBBytes;
+    for (int item = blockIdx.y * blockDim.x + threadIdx.x; item < kBCols + 36 * 32; item += gridDim.y * blockDim.x) {
+        if (item < kBCols) {
+            const int n = item;
+            unsigned char* col = sB + (n >> 3) * 512 + (n & 7) * 16;
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i] = 0u;
+            if (n >= 288) {
+#pragma unroll
+                for (int i = 4; i < 12; ++i) w[i] = kOnesBf16x2;
+                w[12] = pack_bf16(0.f, 1.f); w[13] = pack_bf16(1.f, 0.f);
+            } else {
+                const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;
+                const int cn = n & 31, j = cn >> 3, wi = cn & 7;
+                const float* wc = wvs + (8 * (wi >> 1) + 2 * j + (wi & 1)) * 81 + t;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int s0 = 2 * i, s1 = 2 * i + 1;
+                    w[i] = pack_bf16(wc[s0 * 9] - (s0 == t ? 1.f : 0.f), wc[s1 * 9] - (s1 == t ? 1.f : 0.f));
+                    const uint32_t oh = pack_bf16(s0 == t ? 1.f : 0.f, s1 == t ? 1.f : 0.f);
+                    w[4 + i] = oh; w[8 + i] = oh;
+                }
+                const float o8 = t == 8 ? 1.f : 0.f;
+                w[12] = pack_bf16(wc[72] - o8, o8); w[13] = pack_bf16(o8, 0.f);
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4*>(col + c * 128) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+        } else {
+            const int it = item - kBCols;
+            const int n = it & 31, kg = it >> 5;
+            const int t = kg >> 2, kap0 = (kg & 3) * 8;
+            float val[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int kap = kap0 + e;
+                const int c = 8 * ((kap & 15) >> 2) + (kap & 3) + (kap >= 16 ? 4 : 0);
+                float x = 0.f;
+                if (n < 9) x = wks[c * 81 + n * 9 + t] - (n == t ? 1.f : 0.f);
+                else if (n < 18) x = (n - 9 == t) ? 1.f : 0.f;
+                val[e] = x;
+            }
+            *reinterpret_cast<uint4*>(sBk + kg * 512 + (n >> 3) * 128 + (n & 7) * 16) =
+                make_uint4(pack_bf16(val[0], val[1]), pack_bf16(val[2], val[3]), pack_bf16(val[4], val[5]), pack_bf16(val[6], val[7]));
+        }
+    }
 }
 
 template <int TW>
@@ -150,27 +212,29 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int rank = blockIdx.x / P.heads;
     const int nrank = ((int)gridDim.x - h + P.heads - 1) / P.heads;
     const int tiles_per_head = P.B * P.tiles_y * P.tiles_x;
+    // tiles are dealt round-robin: neighbouring CTAs work on neighbouring tiles at the same time, which
+    // keeps the halos they share in L2
     const int my_tiles = rank < tiles_per_head ? (tiles_per_head - rank + nrank - 1) / nrank : 0;
     const int my_units = my_tiles * U;
     const int my_blocks = (my_units + 3) >> 2;
     const int C = P.heads * kHeadDim;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kKStages; ++s) { mbar_init(bar(kBarKFull + s), 1); mbar_init(bar(kBarKEmpty + s), kPWarps); }
-        for (int s = 0; s < kMaxVStages; ++s) { mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarVEmpty + s), kVWarps); }
-        mbar_init(bar(kBarWeights), 1);
-        mbar_init(bar(kBarWeightsDone), kThreads / 32);
-        for (int i = 0; i < 4; ++i) { mbar_init(bar(kBarPReady + i), kPWarps); mbar_init(bar(kBarPFree + i), 1); }
+        for (int s = 0; s < kKStages; ++s) { mbar_init_only(bar(kBarKFull + s), 1); mbar_init_only(bar(kBarKEmpty + s), kPWarps); }
+        for (int s = 0; s < kMaxVStages; ++s) { mbar_init_only(bar(kBarVFull + s), 1); mbar_init_only(bar(kBarVEmpty + s), kVWarps); }
+        mbar_init_only(bar(kBarWeights), 1);
+        for (int i = 0; i < 4; ++i) { mbar_init_only(bar(kBarPReady + i), kPWarps); mbar_init_only(bar(kBarPFree + i), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(kBarLFull + i), 1);
-            mbar_init(bar(kBarLFree + i), 4);
-            mbar_init(bar(kBarEReady + i), 4);
-            mbar_init(bar(kBarEFree + i), 1);
+            mbar_init_only(bar(kBarLFull + i), 1);
+            mbar_init_only(bar(kBarLFree + i), 4);
+            mbar_init_only(bar(kBarEReady + i), 4);
+            mbar_init_only(bar(kBarEFree + i), 1);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(kBarDFull + i), 1); mbar_init(bar(kBarDFree + i), kVWarps); }
-        mbar_init(bar(kBarVDone), kVWarps);
-        mbar_init(bar(kBarTurn + 0), 1);
-        mbar_init(bar(kBarTurn + 1), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init_only(bar(kBarDFull + i), 1); mbar_init_only(bar(kBarDFree + i), kVWarps); }
+        mbar_init_only(bar(kBarVDone), kVWarps);
+        mbar_init_only(bar(kBarTurn + 0), 1);
+        mbar_init_only(bar(kBarTurn + 1), 1);
+        mbar_init_fence();
     }
     if (warp == kCtlK) tmem_alloc(smem_u32(smem + L.tmem_off), kTmemCols);
     tc_fence_before_sync();
@@ -211,85 +275,29 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     w.tx * TW - 1, w.ty * 4 - 1, w.b);
     };
 
-    // weights are staged in the last V stage; the weights, the first K/q tiles and the first V tiles
-    // are sent for at once
-    const unsigned char* w_stage = smem + L.v_off + (size_t)(SV - 1) * L.halo_pad;
+    // The B images of this CTA's head were laid out by the prep kernel of the same forward; they come
+    // in with one bulk copy, sent for together with the first K/q and V tiles.  Only the MMA threads
+    // wait for them.  The prep kernel may still be running when this kernel starts (programmatic
+    // dependent launch), so the thread that reads its output waits for that grid first; nothing
+    // else in this kernel depends on it.
     int k_issued = 0, v_issued = 0;
     TileWalk kq = walk_begin(), vq = kq;
-    if (my_tiles > 0 && warp == kCtlK && lane == 0) {
-        mbar_expect_tx(bar(kBarWeights), 2 * kWeightBytes);
-        bulk_load_1d(smem_u32(w_stage), P.wk + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
-        bulk_load_1d(smem_u32(w_stage) + kWeightBytes, P.wv + (size_t)h * kHeadDim * 81, kWeightBytes, bar(kBarWeights));
-    }
     if (my_tiles > 0 && warp == kCtlT) {
         // the same lane is elected here and in the refill loop below (the election is deterministic for
         // a given member mask), so the ring positions it advances here are the ones it continues from
         uint32_t leader;
         if (elect_one(leader)) {
             while (k_issued < my_tiles && k_issued < kKStages) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; }
-            while (v_issued < my_tiles && v_issued < SV - 1) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
+            while (v_issued < my_tiles && v_issued < SV) { issue_v_tile(vq); walk_next(vq, SV); ++v_issued; }
         }
     }
-    __syncwarp();
-
-    bool ok = my_tiles > 0 && warp_wait(bar(kBarWeights), 0);
-    const float* wks = reinterpret_cast<const float*>(w_stage);
-    const float* wvs = wks + kHeadDim * 81;
-
-    if (ok) {
-        // ---- value-side B tile: column n = (tap-column-major tap, channel), 64 bytes of K each --------
-        unsigned char* sB = smem + L.b_off;
-        for (int n = threadIdx.x; n < kBCols; n += kThreads) {
-            unsigned char* col = sB + (n >> 3) * 512 + (n & 7) * 16;
-            uint32_t w[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) w[i] = 0u;
-            if (n >= 288) {
-#pragma unroll
-                for (int i = 4; i < 12; ++i) w[i] = kOnesBf16x2;
-                w[12] = pack_bf16(0.f, 1.f); w[13] = pack_bf16(1.f, 0.f);
-            } else {
-                const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;
-                const int cn = n & 31, j = cn >> 3, wi = cn & 7;
-                const float* wc = wvs + (8 * (wi >> 1) + 2 * j + (wi & 1)) * 81 + t;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int s0 = 2 * i, s1 = 2 * i + 1;
-                    w[i] = pack_bf16(wc[s0 * 9] - (s0 == t ? 1.f : 0.f), wc[s1 * 9] - (s1 == t ? 1.f : 0.f));
-                    const uint32_t oh = pack_bf16(s0 == t ? 1.f : 0.f, s1 == t ? 1.f : 0.f);
-                    w[4 + i] = oh; w[8 + i] = oh;
-                }
-                const float o8 = t == 8 ? 1.f : 0.f;
-                w[12] = pack_bf16(wc[72] - o8, o8); w[13] = pack_bf16(o8, 0.f);
-            }
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                *reinterpret_cast<uint4*>(col + c * 128) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-        }
-        // ---- key-side B: [k-group of 8][n-group of 8][8 n rows][8 k] bf16; K index = 32 tap + kappa,
-        // kappa -> channel as the product warps' tcgen05.st lays P out
-        unsigned char* sBk = smem + L.bk_off;
-        for (int item = threadIdx.x; item < 36 * 32; item += kThreads) {
-            const int n = item & 31, kg = item >> 5;
-            const int t = kg >> 2, kap0 = (kg & 3) * 8;
-            float val[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int kap = kap0 + e;
-                const int c = 8 * ((kap & 15) >> 2) + (kap & 3) + (kap >= 16 ? 4 : 0);
-                float x = 0.f;
-                if (n < 9) x = wks[c * 81 + n * 9 + t] - (n == t ? 1.f : 0.f);
-                else if (n < 18) x = (n - 9 == t) ? 1.f : 0.f;
-                val[e] = x;
-            }
-            *reinterpret_cast<uint4*>(sBk + kg * 512 + (n >> 3) * 128 + (n & 7) * 16) =
-                make_uint4(pack_bf16(val[0], val[1]), pack_bf16(val[2], val[3]), pack_bf16(val[4], val[5]), pack_bf16(val[6], val[7]));
-        }
-        fence_proxy_async_smem();
+    if (my_tiles > 0 && warp == kCtlV && lane == 0) {
+        grid_dependency_wait();
+        mbar_expect_tx(bar(kBarWeights), kImgBytes);
+        bulk_load_1d(smem_u32(smem + L.b_off), P.bimg + (size_t)h * kImgBytes, kImgBytes, bar(kBarWeights));
     }
-    __syncthreads();
     __syncwarp();
-    if (lane == 0) mbar_arrive(bar(kBarWeightsDone));
+    bool ok = my_tiles > 0;
 
     if (warp >= kVWarps && warp < kCtlK) {
         // =====================================================================================
@@ -529,6 +537,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // one has got past the P-ready wait of the last chunk of block b - 1, so the P-ready
             // barriers are waited on strictly in chunk order.
             const int me = warp == kCtlK ? 0 : 1;
+            if (!mbar_wait(bar(kBarWeights), 0)) ok = false;
             for (int blk = me, n = 0; ok && blk < my_blocks; blk += 2, ++n) {
                 const int lb = blk & 1;
                 const uint32_t dcol = tmem + kColL + 32 * lb;
@@ -572,6 +581,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const bool elected = elect_one(leader);
         if (elected && ok) {
             const uint32_t sB0 = smem_u32(smem + L.b_off);
+            if (!mbar_wait(bar(kBarWeights), 0)) ok = false;
             for (int blk = 0; ok && blk < my_blocks; ++blk) {
                 const int eb = blk & 1;
                 if (!mbar_wait(bar(kBarEReady + eb), (blk >> 1) & 1)) { ok = false; break; }
@@ -599,17 +609,14 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         uint32_t leader;
         const bool elected = elect_one(leader);
         if (elected && ok) {
-            bool weights_done = false;
             int left = my_tiles - v_issued + my_tiles - k_issued;
             uint32_t idle = 0;
             while (left > 0) {
-                if (!weights_done) weights_done = mbar_test(bar(kBarWeightsDone), 0);
                 const uint32_t tK = mbar_test_u32(bar(kBarKEmpty + kq.stage), (kq.round - 1) & 1);
                 const uint32_t tV = mbar_test_u32(bar(kBarVEmpty + vq.stage), (vq.round - 1) & 1);
                 const int left_before = left;
                 if (tK != 0 && k_issued < my_tiles) { issue_k_tile(kq); walk_next(kq, kKStages); ++k_issued; --left; }
-                // the last V stage held the weights: its first tile waits until every warp is done with them
-                if (tV != 0 && v_issued < my_tiles && (v_issued != SV - 1 || weights_done)) {
+                if (tV != 0 && v_issued < my_tiles) {
                     issue_v_tile(vq); walk_next(vq, SV); ++v_issued; --left;
                 }
                 if (left != left_before) idle = 0;
@@ -622,36 +629,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
     }
     if (!ok && my_tiles > 0 && lane == 0) atomicExch(P.status, 1);
-}
-
-// ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-bool make_map(CUtensorMap* map, const void* base, int B, int H, int W, int C, int bw, int bh) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)bw, (cuuint32_t)bh, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -667,18 +644,32 @@ cudaError_t setup_one() {
     return cudaFuncSetAttribute(umma_ts_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
 }
 
+// The main kernel is launched with programmatic stream serialisation: it may begin (barrier set-up,
+// tensor-memory allocation, first tile loads) while the prep kernel before it in the stream is still
+// running; the one thread that reads the prep kernel's output waits for that grid inside the kernel.
 template <int TW>
 cudaError_t launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& P,
                        int grid, cudaStream_t stream) {
     static_assert(v_stages_for(TW) >= 2, "tile width does not fit shared memory");
-    umma_ts_kernel<TW><<<grid, kThreads, smem_layout(TW, v_stages_for(TW)).total, stream>>>(mq, mk, mv, P);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_layout(TW, v_stages_for(TW)).total;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, umma_ts_kernel<TW>, mq, mk, mv, P);
 }
 
 }  // namespace
 
+size_t umma_ts_workspace_bytes(int heads) { return (size_t)heads * kImgBytes; }
+
 cudaError_t umma_ts_setup() {
-    if (!encode_fn()) return cudaErrorNotSupported;
+    if (!tensor_map_available()) return cudaErrorNotSupported;
     cudaError_t e = setup_one<8>();
     if (e == cudaSuccess) e = setup_one<16>();
     if (e == cudaSuccess) e = setup_one<24>();
@@ -690,11 +681,16 @@ cudaError_t umma_ts_setup() {
     return e;
 }
 
-cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStream_t stream) {
+cudaError_t launch_umma_ts_prep(const Problem& p, void* workspace, cudaStream_t stream) {
+    umma_ts_prep_kernel<<<dim3((unsigned)p.heads, 6), 256, 0, stream>>>(p.wk, p.wv, static_cast<unsigned char*>(workspace));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_umma_ts(const Problem& p, const void* workspace, int* d_status, int num_sms, cudaStream_t stream) {
     const int txn = (p.W + 63) / 64;
     const int TW = ((((p.W + txn - 1) / txn) + 7) / 8) * 8;
     UmmaParams P;
-    P.wk = p.wk; P.wv = p.wv; P.bias = p.bias;
+    P.bimg = static_cast<const unsigned char*>(workspace); P.bias = p.bias;
     P.out = static_cast<__nv_bfloat16*>(p.out);
     P.status = d_status;
     P.B = p.B; P.H = p.H; P.W = p.W; P.heads = p.heads;
@@ -704,9 +700,9 @@ cudaError_t launch_umma_ts(const Problem& p, int* d_status, int num_sms, cudaStr
 
     const int C = p.heads * kHeadDim;
     CUtensorMap map_q, map_k, map_v;
-    if (!make_map(&map_q, p.q, p.B, p.H, p.W, C, TW, 4) ||
-        !make_map(&map_k, p.k, p.B, p.H, p.W, C, TW + 2, 6) ||
-        !make_map(&map_v, p.v, p.B, p.H, p.W, C, TW + 2, 6))
+    if (!make_tile_map(&map_q, p.q, 2, p.B, p.H, p.W, C, kHeadDim, TW, 4) ||
+        !make_tile_map(&map_k, p.k, 2, p.B, p.H, p.W, C, kHeadDim, TW + 2, 6) ||
+        !make_tile_map(&map_v, p.v, 2, p.B, p.H, p.W, C, kHeadDim, TW + 2, 6))
         return cudaErrorInvalidValue;
 
     const long long tiles = (long long)P.tiles_x * P.tiles_y * p.B * p.heads;

@@ -70,12 +70,13 @@ def ncu_traffic(variant, workload):
     return rec["bytes"] if h == rec["sha256"] else None
 
 
-def other_rooflines(cfg, kernel_ms):
+def other_rooflines(cfg, kernel_ms, fixed_shift=False):
     """The method's own arithmetic against the two compute ceilings, for context beside the HBM figure:
-    2 C (2 k^4 + 2 k^2) flops per query pixel; fp32 ALU ceiling = SMs x 128 lanes x 2 x max SM clock;
-    bf16 tensor ceiling = the measured cuBLAS figure (burst)."""
+    2 C (2 k^4 + 2 k^2) flops per query pixel (2 C 2 k^2 with fixed-shift weights); fp32 ALU ceiling =
+    SMs x 128 lanes x 2 x max SM clock; bf16 tensor ceiling = the measured cuBLAS figure (burst)."""
     k2 = cfg["ksize"] ** 2
-    flops = 2.0 * cfg["heads"] * cfg["head_dim"] * (2 * k2 * k2 + 2 * k2) * cfg["B"] * cfg["H"] * cfg["W"]
+    per_channel = 2 * k2 if fixed_shift else 2 * k2 * k2 + 2 * k2
+    flops = 2.0 * cfg["heads"] * cfg["head_dim"] * per_channel * cfg["B"] * cfg["H"] * cfg["W"]
     out = {"flops_per_launch": flops}
     if not kernel_ms or kernel_ms <= 0:
         return out
@@ -306,6 +307,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other", action="store_true", help="skip the kernel-only figures of the other gated shapes")
+    ap.add_argument("--fixed-shift", action="store_true",
+                    help="the workload with exactly one-hot depthwise weights (sigma_w = 0), run in fixed-shift mode")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -328,6 +331,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     cfg = dict(synth.CONFIGS[args.workload])
+    if args.fixed_shift:
+        cfg["sigma_w"] = 0.0
     x = synth.make_inputs(**cfg)
     td = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
     host = {n: torch.from_numpy(x[n]).to(td) for n in ("q", "k", "v")}
@@ -351,6 +356,9 @@ def main():
     if args.variant != "auto":
         sa.slide_attn_set_variant(ctx, VARIANT_IDS[args.variant])
     variant = {v: k for k, v in VARIANT_IDS.items()}[sa.slide_attn_get_variant(ctx)]
+    if args.fixed_shift:
+        sa.slide_attn_set_fixed_shift(ctx, True)
+        variant = "fixed_shift"
     launches = sa.slide_attn_launches_per_forward(ctx)
     stream = torch.cuda.current_stream()
 
@@ -426,7 +434,7 @@ def main():
     sa.slide_attn_destroy(ctx)
 
     other = None
-    if rank == 0 and world == 1 and not args.no_other:
+    if rank == 0 and world == 1 and not args.no_other and not args.fixed_shift:
         vid = 0 if args.variant == "auto" else VARIANT_IDS[args.variant]
         del sets
         torch.cuda.empty_cache()
@@ -457,7 +465,7 @@ def main():
             "timing": {"repeats": len(repeat_ms), "steps_per_repeat": args.steps, "reported": "median repeat",
                        "median_ms_per_step": float(np.median(repeat_ms)), "min_ms_per_step": float(min(repeat_ms)),
                        "max_ms_per_step": float(max(repeat_ms))},
-            "compute_ceilings": other_rooflines(cfg, main_ms),
+            "compute_ceilings": other_rooflines(cfg, main_ms, args.fixed_shift),
             "clocks": clocks, "e2e": e2e,
         }
         if world == 1 and not args.no_cpu_baseline:

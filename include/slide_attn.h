@@ -70,7 +70,9 @@ typedef enum {
     SLIDE_ATTN_ERR_CUDA        = 5,   /* a CUDA runtime/driver call failed                         */
     SLIDE_ATTN_ERR_ARCH        = 6,   /* current device is not compute capability 10.x             */
     SLIDE_ATTN_ERR_TIMEOUT     = 7,   /* a bounded device-side wait ran out (see query_status)     */
-    SLIDE_ATTN_ERR_TOO_LARGE   = 8    /* problem exceeds the fixed scratch of forward_noalloc      */
+    SLIDE_ATTN_ERR_TOO_LARGE   = 8,   /* problem exceeds the fixed scratch of forward_noalloc      */
+    SLIDE_ATTN_ERR_NOT_FIXED_SHIFT = 9 /* fixed-shift mode was declared but a weight is not one-hot
+                                          (reported by query_status; that forward's output is undefined) */
 } slide_attn_status;
 
 /* Kernel variants.  AUTO picks the fastest one that supports the context's shape; the others
@@ -155,12 +157,35 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* ctx, slide_attn_variant
 /* The variant the next forward will run (never AUTO).  *variant [out, host]. */
 slide_attn_status slide_attn_get_variant(const slide_attn_ctx* ctx, slide_attn_variant* variant);
 
+/*
+ * Fixed-shift mode (Sec. 4.2, Eq. 8-13; the "shift" / depthwise-convolution forms of the method
+ * without the deformed shifting module of Sec. 4.3).  With enable != 0 the caller declares that the
+ * wk and wv given to later forwards are EXACTLY the one-hot shift kernels of Eq. 11
+ * (w[c][s][t] = 1 if t == s, else 0).  Slot s of a pixel then is the key / value at window offset s,
+ * and the forward runs a kernel that does 2 k^2 instead of 2 k^4 + 2 k^2 multiply-adds per
+ * pixel-channel (head_dim 32, ksize <= 9, both dtypes; SLIDE_ATTN_ERR_UNSUPPORTED otherwise, and the
+ * mode stays off).  Every forward in this mode still reads wk and wv once on the device and checks the
+ * declaration: if a weight differs, the status word is set and the next slide_attn_query_status
+ * returns SLIDE_ATTN_ERR_NOT_FIXED_SHIFT; that forward's output is undefined.  enable == 0 returns to
+ * the general kernels.  slide_attn_set_variant has no effect while the mode is on.
+ */
+slide_attn_status slide_attn_set_fixed_shift(slide_attn_ctx* ctx, int enable);
+
+/*
+ * Tells whether wk and wv (DEVICE, float [C][k*k][k*k]) are exactly the one-hot shift kernels of
+ * Eq. 11, so that a caller can decide on fixed-shift mode when it loads a model.  Runs a reduction
+ * on `cuda_stream` and WAITS for it.  *is_fixed [out, host] = 1 or 0.
+ */
+slide_attn_status slide_attn_detect_fixed_shift(slide_attn_ctx* ctx, const float* wk, const float* wv,
+                                                int* is_fixed, void* cuda_stream);
+
 /* Number of kernels one slide_attn_forward launches with the current variant.  *n [out, host]. */
 slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* ctx, int* n);
 
 /*
- * Waits for `cuda_stream` and reports the device-side status word: SLIDE_ATTN_OK, or
- * SLIDE_ATTN_ERR_TIMEOUT if a kernel gave up on a bounded wait (its output is then undefined).
+ * Waits for `cuda_stream` and reports the device-side status word: SLIDE_ATTN_OK,
+ * SLIDE_ATTN_ERR_TIMEOUT if a kernel gave up on a bounded wait, or SLIDE_ATTN_ERR_NOT_FIXED_SHIFT if a
+ * forward in fixed-shift mode met a weight that is not one-hot (the output is then undefined).
  * The word is cleared by this call.
  */
 slide_attn_status slide_attn_query_status(slide_attn_ctx* ctx, void* cuda_stream);

@@ -18,10 +18,12 @@ F32, BF16 = 0, 1
 VARIANT_AUTO, VARIANT_DIRECT, VARIANT_MMA, VARIANT_MMA_WS, VARIANT_UMMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_UMMA_SP = 0, 1, 2, 3, 4, 5, 6, 7
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(8)
 ERR_TOO_LARGE = 8
+ERR_NOT_FIXED_SHIFT = 9
 
 EXPORTS = ("slide_attn_create", "slide_attn_forward", "slide_attn_forward_host",
            "slide_attn_forward_noalloc",
            "slide_attn_set_variant", "slide_attn_get_variant", "slide_attn_launches_per_forward",
+           "slide_attn_set_fixed_shift", "slide_attn_detect_fixed_shift",
            "slide_attn_profile_begin", "slide_attn_profile_end",
            "slide_attn_query_status", "slide_attn_destroy", "slide_attn_status_string")
 
@@ -50,6 +52,8 @@ def load() -> ctypes.CDLL:
         lib.slide_attn_forward_noalloc.argtypes = [vp] * 7 + [i] * 7 + [vp]
         lib.slide_attn_set_variant.argtypes = [vp, i]
         lib.slide_attn_get_variant.argtypes = [vp, ctypes.POINTER(i)]
+        lib.slide_attn_set_fixed_shift.argtypes = [vp, i]
+        lib.slide_attn_detect_fixed_shift.argtypes = [vp, vp, vp, ctypes.POINTER(i), vp]
         lib.slide_attn_launches_per_forward.argtypes = [vp, ctypes.POINTER(i)]
         lib.slide_attn_profile_begin.argtypes = [vp]
         lib.slide_attn_profile_end.argtypes = [vp, ctypes.POINTER(ctypes.c_double),
@@ -134,6 +138,20 @@ def slide_attn_set_variant(ctx, variant: int) -> None:
     _check(load().slide_attn_set_variant(ctx, int(variant)), "slide_attn_set_variant")
 
 
+def slide_attn_set_fixed_shift(ctx, enable: bool) -> None:
+    """Declares that later forwards get exactly the one-hot shift kernels as wk and wv (checked on
+    the device in every forward); they then run the fixed-shift kernel."""
+    _check(load().slide_attn_set_fixed_shift(ctx, int(bool(enable))), "slide_attn_set_fixed_shift")
+
+
+def slide_attn_detect_fixed_shift(ctx, wk, wv, stream=None) -> bool:
+    """True if the device tensors wk and wv are exactly the one-hot shift kernels (synchronises)."""
+    r = ctypes.c_int()
+    _check(load().slide_attn_detect_fixed_shift(ctx, _dev_ptr(wk), _dev_ptr(wv), ctypes.byref(r), _stream_ptr(stream)),
+           "slide_attn_detect_fixed_shift")
+    return bool(r.value)
+
+
 def slide_attn_get_variant(ctx) -> int:
     v = ctypes.c_int()
     _check(load().slide_attn_get_variant(ctx, ctypes.byref(v)), "slide_attn_get_variant")
@@ -161,7 +179,7 @@ def slide_attn_profile_end(ctx):
 def slide_attn_query_status(ctx, stream=None) -> int:
     """Synchronises the stream; returns OK or ERR_TIMEOUT (does not raise on timeout)."""
     st = load().slide_attn_query_status(ctx, _stream_ptr(stream))
-    if st not in (OK, ERR_TIMEOUT):
+    if st not in (OK, ERR_TIMEOUT, ERR_NOT_FIXED_SHIFT):
         raise SlideAttnError(st, "slide_attn_query_status")
     return st
 

@@ -78,6 +78,13 @@ size_t umma_ts_workspace_bytes(int heads);
 cudaError_t launch_umma_ts_prep(const Problem& p, void* workspace, cudaStream_t stream);
 cudaError_t launch_umma_ts(const Problem& p, const void* workspace, int* d_status, int num_sms, cudaStream_t stream);
 
+// Fixed-shift fast path: plain k x k local attention for weights that are exactly the one-hot shift
+// kernels (head_dim 32, k <= 9, fp32 or bf16).  launch_shift_check sets the status word to 2 when a
+// weight differs from the one-hot kernel.
+bool shift_supports(int head_dim, int ksize);
+cudaError_t launch_shift_check(const Problem& p, int* d_status, cudaStream_t stream);
+cudaError_t launch_shift(const Problem& p, int* d_status, cudaStream_t stream);
+
 // UMMA_SP variant: the tcgen05 arithmetic of UMMA_TS in ONE software-pipelined team of eight warps
 // (every warp forms q.k products, takes its turn at the softmax and applies the value weights), so
 // tensor memory is single-buffered and a block costs four barrier hand-offs instead of twenty.

@@ -10,6 +10,7 @@ struct slide_attn_ctx {
     int B, H, W, heads, head_dim, ksize, has_bias;
     slide_attn_dtype dtype;
     slide_attn_variant variant;      // never AUTO
+    bool fixed_shift;                // the caller declared one-hot weights: run the fixed-shift kernel
     int device;
     int num_sms;
     int* d_status;                   // device status word (0 = ok)
@@ -90,6 +91,13 @@ slide_attn_status launch_problem(slide_attn_ctx* c, const Problem& p, cudaStream
         cudaEventRecord(ev[0], stream);
     }
     cudaError_t err;
+    if (c->fixed_shift) {
+        err = launch_shift_check(p, c->d_status, stream);
+        if (ev) cudaEventRecord(ev[1], stream);
+        if (err == cudaSuccess) err = launch_shift(p, c->d_status, stream);
+        if (ev) { cudaEventRecord(ev[2], stream); c->prof_count++; }
+        return err == cudaSuccess ? SLIDE_ATTN_OK : SLIDE_ATTN_ERR_CUDA;
+    }
     switch (c->variant) {
         case SLIDE_ATTN_VARIANT_DIRECT:
             if (ev) cudaEventRecord(ev[1], stream);
@@ -320,6 +328,37 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant v
     return SLIDE_ATTN_OK;
 }
 
+slide_attn_status slide_attn_set_fixed_shift(slide_attn_ctx* c, int enable)
+{
+    if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (enable && !shift_supports(c->head_dim, c->ksize)) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    c->fixed_shift = enable != 0;
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_detect_fixed_shift(slide_attn_ctx* c, const float* wk, const float* wv,
+                                                int* is_fixed, void* cuda_stream)
+{
+    if (!c || !wk || !wv || !is_fixed) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // a word of its own is not needed: the context's status word is read, used and restored in
+    // stream order, and the call waits for all of it
+    int before = 0, after = 0;
+    Problem p = {};
+    p.heads = c->heads; p.head_dim = c->head_dim; p.ksize = c->ksize; p.wk = wk; p.wv = wv;
+    bool ok = cudaMemcpyAsync(&before, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaMemsetAsync(c->d_status, 0, sizeof(int), stream) == cudaSuccess &&
+              launch_shift_check(p, c->d_status, stream) == cudaSuccess &&
+              cudaMemcpyAsync(&after, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaStreamSynchronize(stream) == cudaSuccess;
+    if (ok) ok = cudaMemcpyAsync(c->d_status, &before, sizeof(int), cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+                 cudaStreamSynchronize(stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+    *is_fixed = after == 0 ? 1 : 0;
+    return SLIDE_ATTN_OK;
+}
+
 slide_attn_status slide_attn_get_variant(const slide_attn_ctx* c, slide_attn_variant* variant)
 {
     if (!c || !variant) return SLIDE_ATTN_ERR_INVALID_ARG;
@@ -330,6 +369,7 @@ slide_attn_status slide_attn_get_variant(const slide_attn_ctx* c, slide_attn_var
 slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* n)
 {
     if (!c || !n) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (c->fixed_shift) { *n = 2; return SLIDE_ATTN_OK; }   // weight check + fixed-shift kernel
     switch (c->variant) {
         case SLIDE_ATTN_VARIANT_DIRECT: *n = 1; break;
         case SLIDE_ATTN_VARIANT_MMA: *n = 2; break;      // weight re-layout + fused kernel
@@ -399,7 +439,7 @@ slide_attn_status slide_attn_query_status(slide_attn_ctx* c, void* cuda_stream)
         cudaGetLastError();
         return SLIDE_ATTN_ERR_CUDA;
     }
-    return word == 0 ? SLIDE_ATTN_OK : SLIDE_ATTN_ERR_TIMEOUT;
+    return word == 0 ? SLIDE_ATTN_OK : (word == 2 ? SLIDE_ATTN_ERR_NOT_FIXED_SHIFT : SLIDE_ATTN_ERR_TIMEOUT);
 }
 
 slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
@@ -437,6 +477,7 @@ const char* slide_attn_status_string(slide_attn_status status)
         case SLIDE_ATTN_ERR_ARCH: return "device is not sm_100 (B200)";
         case SLIDE_ATTN_ERR_TIMEOUT: return "device-side wait timed out";
         case SLIDE_ATTN_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of slide_attn_forward_noalloc (16 heads)";
+        case SLIDE_ATTN_ERR_NOT_FIXED_SHIFT: return "fixed-shift mode, but a weight is not the one-hot shift kernel";
         default: return "unknown status";
     }
 }

@@ -29,8 +29,8 @@ def test_library_exports_every_declared_symbol(lib):
 
 
 def test_status_strings(lib):
-    seen = {sa.slide_attn_status_string(s) for s in range(9)}
-    assert len(seen) == 9 and "ok" in seen and "unknown status" not in seen
+    seen = {sa.slide_attn_status_string(s) for s in range(10)}
+    assert len(seen) == 10 and "ok" in seen and "unknown status" not in seen
     assert sa.slide_attn_status_string(99) == "unknown status"
 
 

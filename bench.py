@@ -32,7 +32,7 @@ from paper_2304_04237_b200 import synth  # noqa: E402
 METRIC = "slide_attn_fwd_query_pixels_per_s"
 UNIT = "query-pixels/s"
 FALLBACK_HBM_GBS = 6650.0
-VARIANT_IDS = {"direct": 1, "mma": 2, "mma_ws": 3, "umma": 4, "umma_ts": 5, "strip": 6, "umma_sp": 7}
+VARIANT_IDS = {"direct": 1, "mma": 2, "umma_ts": 5, "strip": 6, "tile": 8}
 
 
 def algorithmic_bytes(cfg) -> int:
@@ -52,9 +52,6 @@ NCU_TRAFFIC = {
     ("umma_ts", "c2"): {"bytes": 82.20e6,
                         "sources": ("paper_2304_04237_b200/csrc/umma_ts_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
                         "sha256": "d2776bf13a3878cd21398729ce2c7985d50bca3179a18d8a15a6041c7fd69bd7"},
-    ("umma", "c2"): {"bytes": 82.36e6,
-                     "sources": ("paper_2304_04237_b200/csrc/umma_kernel.cu", "paper_2304_04237_b200/csrc/ptx.cuh"),
-                     "sha256": "e6187f91a3111cecdd746131ef0e72057c2aa4244a0aab58edba8035ca0a52c9"},
 }
 
 
@@ -302,7 +299,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
-    ap.add_argument("--variant", default="auto", choices=["auto", "direct", "mma", "mma_ws", "umma", "umma_ts", "strip", "umma_sp"])
+    ap.add_argument("--variant", default="auto", choices=["auto"] + sorted(VARIANT_IDS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -76,30 +76,27 @@ typedef enum {
 } slide_attn_status;
 
 /* Kernel variants.  AUTO picks the fastest one that supports the context's shape; the others
- * exist for A/B measurements and tests.  All variants compute the same function. */
+ * exist for A/B measurements and tests.  All variants compute the same function.  (Values 3, 4 and 7
+ * belonged to earlier tensor-core schedules that UMMA_TS replaced; they are not accepted any more.) */
 typedef enum {
     SLIDE_ATTN_VARIANT_AUTO    = 0,
     SLIDE_ATTN_VARIANT_DIRECT  = 1,   /* one warp per (pixel, head), global loads, fp32 FMA; any shape */
     SLIDE_ATTN_VARIANT_MMA     = 2,   /* TMA halo tile in shared memory, deformed-shift contraction on
-                                         tensor cores (bf16 operands, fp32 accumulate); one CTA per
-                                         tile and head; bf16, head_dim 32, ksize 3                      */
-    SLIDE_ATTN_VARIANT_MMA_WS  = 3,   /* same arithmetic, persistent warp-specialised schedule (key
-                                         warps / value warps, 3-stage TMA ring, weights resident in
-                                         registers, single launch); bf16, head_dim 32, ksize 3          */
-    SLIDE_ATTN_VARIANT_UMMA    = 4,   /* MMA_WS with the value-side contraction on the 5th-generation
-                                         tensor core (tcgen05.mma, accumulator in tensor memory);
-                                         bf16, head_dim 32, ksize 3                                     */
-    SLIDE_ATTN_VARIANT_UMMA_TS = 5,   /* both contractions on tcgen05.mma with their A operands (the
-                                         q.k products, the softmax weights) held in tensor memory;
-                                         bf16, head_dim 32, ksize 3                                     */
+                                         mma.sync tensor cores (bf16 operands, fp32 accumulate); one CTA
+                                         per tile and head; bf16, head_dim 32, ksize 3; also what the
+                                         allocation-free entry point runs                              */
+    SLIDE_ATTN_VARIANT_UMMA_TS = 5,   /* persistent warp-specialised kernel, both contractions on
+                                         tcgen05.mma with their A operands (the q.k products, the softmax
+                                         weights) held in tensor memory; bf16, head_dim 32, ksize 3: what
+                                         AUTO runs there                                               */
     SLIDE_ATTN_VARIANT_STRIP   = 6,   /* DIRECT's arithmetic with transposed weights (one coalesced load
-                                         per weight) and 4-8 pixels per warp; fp32 FMA; ksize <= 9,
-                                         any head_dim, fp32 or bf16: what AUTO runs where the tensor-core
-                                         variants do not apply                                          */
-    SLIDE_ATTN_VARIANT_UMMA_SP = 7    /* UMMA_TS's arithmetic as one team of eight warps running a
-                                         software pipeline over the pixel blocks (products, softmax and
-                                         value phase of three consecutive blocks per iteration), tensor
-                                         memory single-buffered; bf16, head_dim 32, ksize 3             */
+                                         per weight) and 4-8 pixels per warp, operands read from global
+                                         memory; fp32 FMA; ksize <= 9, any head_dim, fp32 or bf16        */
+    SLIDE_ATTN_VARIANT_TILE    = 8    /* generic weights on the CUDA cores off a TMA-staged halo tile
+                                         in shared memory, 16-byte accesses throughout, convolution
+                                         re-associated with the q.k products and the softmax weights;
+                                         head_dim 32, ksize <= 9, fp32 or bf16: what AUTO runs where
+                                         UMMA_TS does not apply                                          */
 } slide_attn_variant;
 
 /*

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libslide_attn.so")
 
 F32, BF16 = 0, 1
-VARIANT_AUTO, VARIANT_DIRECT, VARIANT_MMA, VARIANT_MMA_WS, VARIANT_UMMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_UMMA_SP = 0, 1, 2, 3, 4, 5, 6, 7
+VARIANT_AUTO, VARIANT_DIRECT, VARIANT_MMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_TILE = 0, 1, 2, 5, 6, 8
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(8)
 ERR_TOO_LARGE = 8
 ERR_NOT_FIXED_SHIFT = 9

@@ -59,17 +59,6 @@ cudaError_t launch_mma_prep(const Problem& p, void* workspace, cudaStream_t stre
 cudaError_t launch_mma_main(const Problem& p, const void* workspace, int* d_status, cudaStream_t stream);
 
 
-// MMA_WS variant: persistent warp-specialised kernel, single launch, no workspace.
-bool mma_ws_supports(slide_attn_dtype dtype, int head_dim, int ksize);
-cudaError_t mma_ws_setup();
-cudaError_t launch_mma_ws(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
-
-
-// UMMA variant: as MMA_WS, with the value-side contraction on tcgen05 / tensor memory.
-bool umma_supports(slide_attn_dtype dtype, int head_dim, int ksize);
-cudaError_t umma_setup();
-cudaError_t launch_umma(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
-
 // UMMA_TS variant: both contractions on tcgen05 with their A operands in tensor memory.  A prep launch
 // writes the bf16 B images of every head (umma_ts_workspace_bytes) that the main launch's CTAs copy in.
 bool umma_ts_supports(slide_attn_dtype dtype, int head_dim, int ksize);
@@ -85,11 +74,9 @@ bool shift_supports(int head_dim, int ksize);
 cudaError_t launch_shift_check(const Problem& p, int* d_status, cudaStream_t stream);
 cudaError_t launch_shift(const Problem& p, int* d_status, cudaStream_t stream);
 
-// UMMA_SP variant: the tcgen05 arithmetic of UMMA_TS in ONE software-pipelined team of eight warps
-// (every warp forms q.k products, takes its turn at the softmax and applies the value weights), so
-// tensor memory is single-buffered and a block costs four barrier hand-offs instead of twenty.
-bool umma_sp_supports(slide_attn_dtype dtype, int head_dim, int ksize);
-cudaError_t umma_sp_setup();
-cudaError_t launch_umma_sp(const Problem& p, int* d_status, int num_sms, cudaStream_t stream);
+// TILE variant: generic weights, CUDA cores, TMA-staged halo tiles (head_dim 32, k <= 9, both dtypes).
+// Reads the transposed weights that launch_strip_prep writes.
+bool tile_supports(int head_dim, int ksize);
+cudaError_t launch_tile(const Problem& p, const void* workspace, int* d_status, cudaStream_t stream);
 
 }  // namespace slide_attn

@@ -303,34 +303,9 @@ mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CU
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // [B][H][W][C] bf16 viewed as a 4-D tensor (C, W, H, B); box = 32 channels x (TW+2) x (TH+2) x 1.
 bool make_halo_map(CUtensorMap* map, const void* base, int B, int H, int W, int C, int TH, int TW) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)(TW + 2), (cuuint32_t)(TH + 2), 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return make_tile_map(map, base, 2, B, H, W, C, kHeadDim, TW + 2, TH + 2);
 }
 
 void pick_tile(int H, int W, int* TH, int* TW, int* tiles_x, int* tiles_y) {
@@ -357,7 +332,7 @@ size_t mma_workspace_bytes(int heads) { return (size_t)heads * kFragWordsPerHead
 // Per device, once: allow the main kernel its dynamic shared memory and resolve the driver
 // entry point used to encode tensor maps.
 cudaError_t mma_setup() {
-    if (!encode_fn()) return cudaErrorNotSupported;
+    if (!tensor_map_available()) return cudaErrorNotSupported;
     return cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
 }
 

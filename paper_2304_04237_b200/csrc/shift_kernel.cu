@@ -19,103 +19,14 @@
 // column dx the warp walks the 4 + k - 1 halo rows of that column once: each row vector serves every
 // pixel of the strip whose window holds it.  The softmax runs online over the window columns (running
 // maximum, sum and accumulator per pixel), so registers do not grow with k^2.
-#include "common.cuh"
-#include "ptx.cuh"
+#include "tile_common.cuh"
 
 namespace slide_attn {
 
 namespace {
 
-constexpr int kHeadDim = 32;
-constexpr int kTW = 32;                        // tile width in pixels
-constexpr int kR = 4;                          // pixel rows per warp
-constexpr float kLog2e = 1.4426950408889634f;
-
-template <typename T> struct Elem;
-template <> struct Elem<__nv_bfloat16> { static constexpr int planes = 1, th = 4; };
-template <> struct Elem<float> { static constexpr int planes = 2, th = 4; };
-
-template <typename T, int K>
-struct Cfg {
-    static constexpr int planes = Elem<T>::planes;
-    static constexpr int TH = Elem<T>::th;
-    static constexpr int warps = (kTW / 8) * (TH / kR);
-    static constexpr int threads = warps * 32;
-    static constexpr int HW = kTW + K - 1, HH = TH + K - 1;                 // halo tile
-    static constexpr uint32_t halo_plane = (uint32_t)(HW * HH * 64 + 127) & ~127u;
-    static constexpr uint32_t q_plane = (uint32_t)(kTW * TH * 64);
-    static constexpr uint32_t k_off = 0, v_off = planes * halo_plane, q_off = 2 * planes * halo_plane;
-    static constexpr uint32_t bias_off = q_off + planes * q_plane;
-    static constexpr uint32_t bar_off = bias_off + ((K * K * 4 + 15) & ~15);
-    static constexpr uint32_t total = bar_off + 16 + 128;                   // + alignment slack
-    static constexpr uint32_t tx_bytes = planes * (2u * HW * HH * 64u + q_plane);
-};
-
-struct ShiftParams {
-    const float* bias;
-    void* out;
-    int* status;
-    int B, H, W, heads;
-    int tiles_x, tiles_y;
-    float scale_log2e;
-};
-
-// Eight channels of one pixel (the piece of lane tig), as loaded and as floats.  bf16: one 16-byte load,
-// kept packed for the q.k products (bf16 x bf16 + fp32 in one instruction, exact products) and widened
-// for the value side; fp32: one 16-byte load per plane.
-template <typename T> struct Piece;
-template <> struct Piece<__nv_bfloat16> {
-    struct Raw { uint32_t w[4]; };
-    static __device__ __forceinline__ Raw load(const unsigned char* tile, uint32_t plane_bytes, uint32_t pix, int tig) {
-        const uint4 v = *reinterpret_cast<const uint4*>(tile + pix * 64u + tig * 16u);
-        Raw r; r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w;
-        return r;
-    }
-    static __device__ __forceinline__ float dot(const Raw& a, const Raw& b) {
-        float acc = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
-                "mov.b32 {al, ah}, %1;\n\tmov.b32 {bl, bh}, %2;\n\t"
-                "fma.rn.f32.bf16 %0, al, bl, %0;\n\t"
-                "fma.rn.f32.bf16 %0, ah, bh, %0;\n\t}"
-                : "+f"(acc) : "r"(a.w[i]), "r"(b.w[i]));
-        return acc;
-    }
-    static __device__ __forceinline__ void widen(const Raw& r, float (&f)[8]) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { f[2 * i] = bf16_lo(r.w[i]); f[2 * i + 1] = bf16_hi(r.w[i]); }
-    }
-};
-template <> struct Piece<float> {
-    struct Raw { float f[8]; };
-    static __device__ __forceinline__ Raw load(const unsigned char* tile, uint32_t plane_bytes, uint32_t pix, int tig) {
-        const float4 a = *reinterpret_cast<const float4*>(tile + pix * 64u + tig * 16u);
-        const float4 b = *reinterpret_cast<const float4*>(tile + plane_bytes + pix * 64u + tig * 16u);
-        Raw r;
-        r.f[0] = a.x; r.f[1] = a.y; r.f[2] = a.z; r.f[3] = a.w; r.f[4] = b.x; r.f[5] = b.y; r.f[6] = b.z; r.f[7] = b.w;
-        return r;
-    }
-    static __device__ __forceinline__ float dot(const Raw& a, const Raw& b) {
-        float p0 = a.f[0] * b.f[0], p1 = a.f[1] * b.f[1];
-        ffma2(p0, p1, a.f[2], a.f[3], b.f[2], b.f[3]);
-        ffma2(p0, p1, a.f[4], a.f[5], b.f[4], b.f[5]);
-        ffma2(p0, p1, a.f[6], a.f[7], b.f[6], b.f[7]);
-        return p0 + p1;
-    }
-    static __device__ __forceinline__ void widen(const Raw& r, float (&f)[8]) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) f[i] = r.f[i];
-    }
-};
-
-__device__ __forceinline__ void fmul2(float& a0, float& a1, float b0, float b1) {
-    asm("{\n\t.reg .b64 ra, rb;\n\t"
-        "mov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
-        "mul.rn.f32x2 ra, ra, rb;\n\t"
-        "mov.b64 {%0, %1}, ra;\n\t}"
-        : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
-}
+using namespace tile;
+using ShiftParams = TileParams;
 
 template <typename T, int K>
 __global__ void __launch_bounds__(Cfg<T, K>::threads, (sizeof(T) == 2 && K <= 3) ? 6 : 4)
@@ -297,7 +208,7 @@ cudaError_t launch_t(const Problem& p, int* d_status, cudaStream_t stream) {
         if (e != cudaSuccess) return e;
     }
     ShiftParams P;
-    P.bias = p.bias; P.out = p.out; P.status = d_status;
+    P.wt = nullptr; P.bias = p.bias; P.out = p.out; P.status = d_status;
     P.B = p.B; P.H = p.H; P.W = p.W; P.heads = p.heads;
     P.tiles_x = (p.W + kTW - 1) / kTW;
     P.tiles_y = (p.H + C_::TH - 1) / C_::TH;

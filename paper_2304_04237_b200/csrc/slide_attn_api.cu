@@ -52,18 +52,15 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
         case SLIDE_ATTN_VARIANT_DIRECT: return direct_supports(c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_STRIP: return c->strip_ws && strip_supports(c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_MMA: return c->workspace && mma_supports(c->dtype, c->head_dim, c->ksize);
-        case SLIDE_ATTN_VARIANT_MMA_WS: return mma_ws_supports(c->dtype, c->head_dim, c->ksize);
-        case SLIDE_ATTN_VARIANT_UMMA: return umma_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA_TS: return c->umma_ws && umma_ts_supports(c->dtype, c->head_dim, c->ksize);
-        case SLIDE_ATTN_VARIANT_UMMA_SP: return umma_sp_supports(c->dtype, c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_TILE: return c->strip_ws && tile_supports(c->head_dim, c->ksize);
         default: return false;
     }
 }
 
 slide_attn_variant pick_variant(const slide_attn_ctx* c) {
-    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA_TS, SLIDE_ATTN_VARIANT_UMMA, SLIDE_ATTN_VARIANT_MMA_WS,
-                                        SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_STRIP,
-                                        SLIDE_ATTN_VARIANT_DIRECT};
+    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA_TS, SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_TILE,
+                                        SLIDE_ATTN_VARIANT_STRIP, SLIDE_ATTN_VARIANT_DIRECT};
     for (slide_attn_variant v : order)
         if (variant_supported(c, v)) return v;
     return SLIDE_ATTN_VARIANT_DIRECT;
@@ -113,22 +110,15 @@ slide_attn_status launch_problem(slide_attn_ctx* c, const Problem& p, cudaStream
             if (ev) cudaEventRecord(ev[1], stream);
             if (err == cudaSuccess) err = launch_mma_main(p, c->workspace, c->d_status, stream);
             break;
-        case SLIDE_ATTN_VARIANT_MMA_WS:
-            if (ev) cudaEventRecord(ev[1], stream);
-            err = launch_mma_ws(p, c->d_status, c->num_sms, stream);
-            break;
-        case SLIDE_ATTN_VARIANT_UMMA:
-            if (ev) cudaEventRecord(ev[1], stream);
-            err = launch_umma(p, c->d_status, c->num_sms, stream);
-            break;
         case SLIDE_ATTN_VARIANT_UMMA_TS:
             err = launch_umma_ts_prep(p, c->umma_ws, stream);
             if (ev) cudaEventRecord(ev[1], stream);
             if (err == cudaSuccess) err = launch_umma_ts(p, c->umma_ws, c->d_status, c->num_sms, stream);
             break;
-        case SLIDE_ATTN_VARIANT_UMMA_SP:
+        case SLIDE_ATTN_VARIANT_TILE:
+            err = launch_strip_prep(p, c->strip_ws, stream);
             if (ev) cudaEventRecord(ev[1], stream);
-            err = launch_umma_sp(p, c->d_status, c->num_sms, stream);
+            if (err == cudaSuccess) err = launch_tile(p, c->strip_ws, c->d_status, stream);
             break;
         default: return SLIDE_ATTN_ERR_UNSUPPORTED;
     }
@@ -181,8 +171,7 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
         return SLIDE_ATTN_ERR_ALLOC;
     }
     if (mma_supports(dtype, head_dim, ksize)) {
-        if (mma_setup() != cudaSuccess || mma_ws_setup() != cudaSuccess || umma_setup() != cudaSuccess ||
-            umma_ts_setup() != cudaSuccess || umma_sp_setup() != cudaSuccess) {
+        if (mma_setup() != cudaSuccess || umma_ts_setup() != cudaSuccess) {
             cudaGetLastError();
             slide_attn_destroy(c);
             return SLIDE_ATTN_ERR_CUDA;
@@ -321,7 +310,8 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant v
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (variant == SLIDE_ATTN_VARIANT_AUTO) { c->variant = pick_variant(c); return SLIDE_ATTN_OK; }
-    if (variant < SLIDE_ATTN_VARIANT_AUTO || variant > SLIDE_ATTN_VARIANT_UMMA_SP)
+    if (variant != SLIDE_ATTN_VARIANT_DIRECT && variant != SLIDE_ATTN_VARIANT_MMA && variant != SLIDE_ATTN_VARIANT_UMMA_TS &&
+        variant != SLIDE_ATTN_VARIANT_STRIP && variant != SLIDE_ATTN_VARIANT_TILE)
         return SLIDE_ATTN_ERR_INVALID_ARG;
     if (!variant_supported(c, variant)) return SLIDE_ATTN_ERR_UNSUPPORTED;
     c->variant = variant;
@@ -374,10 +364,8 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
         case SLIDE_ATTN_VARIANT_DIRECT: *n = 1; break;
         case SLIDE_ATTN_VARIANT_MMA: *n = 2; break;      // weight re-layout + fused kernel
         case SLIDE_ATTN_VARIANT_STRIP: *n = 2; break;    // weight transpose + fused kernel
-        case SLIDE_ATTN_VARIANT_MMA_WS: *n = 1; break;
-        case SLIDE_ATTN_VARIANT_UMMA: *n = 1; break;
         case SLIDE_ATTN_VARIANT_UMMA_TS: *n = 2; break;  // B-image prep + fused kernel
-        case SLIDE_ATTN_VARIANT_UMMA_SP: *n = 1; break;
+        case SLIDE_ATTN_VARIANT_TILE: *n = 2; break;     // weight transpose + fused kernel
         default: *n = 1; break;
     }
     return SLIDE_ATTN_OK;

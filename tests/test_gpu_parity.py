@@ -15,8 +15,8 @@ from util import TORCH_DTYPE, VARIANTS, assert_close, gpu_forward, to_device
 
 pytestmark = pytest.mark.gpu
 
-ALL_VARIANTS = ["auto", "direct", "strip", "mma", "mma_ws", "umma", "umma_ts", "umma_sp"]
-PIPELINED = ["mma_ws", "umma", "umma_ts", "umma_sp"]
+ALL_VARIANTS = ["auto", "direct", "strip", "tile", "mma", "umma_ts"]
+PIPELINED = ["umma_ts"]
 
 
 def ref_forward(x, k):

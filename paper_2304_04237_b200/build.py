@@ -68,5 +68,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_probes() -> list:
+    """Compiles the stand-alone measurement programs of probes/ (not part of the library)."""
+    src_dir = os.path.join(HERE, "probes")
+    out_dir = os.path.join(src_dir, "_build")
+    os.makedirs(out_dir, exist_ok=True)
+    outs = []
+    for s in sorted(glob.glob(os.path.join(src_dir, "*.cu"))):
+        exe = os.path.join(out_dir, os.path.basename(s)[:-3])
+        r = subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+                            "-I", CSRC, "-I", os.path.join(ROOT, "include"), s, "-o", exe], capture_output=True, text=True)
+        if r.returncode != 0:
+            sys.stderr.write(r.stdout + r.stderr)
+            raise RuntimeError("nvcc failed for " + s)
+        outs.append(exe)
+    return outs
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--probes" in sys.argv:
+        print("\n".join(build_probes()))

@@ -307,6 +307,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other", action="store_true", help="skip the kernel-only figures of the other gated shapes")
+    ap.add_argument("--backward", type=int, default=0, metavar="N",
+                    help="also time N backward passes (slide_attn_backward) of the workload and report them beside the forward")
     ap.add_argument("--fixed-shift", action="store_true",
                     help="the workload with exactly one-hot depthwise weights (sigma_w = 0), run in fixed-shift mode")
     args = ap.parse_args()
@@ -410,6 +412,29 @@ def main():
     fwd_ms, main_ms, n_prof = kernel_pass(min(max(args.steps, 200), 1000), step)
     assert sa.slide_attn_query_status(ctx) == sa.OK
 
+    # optional: the backward pass of the same workload (gradients of all six inputs)
+    backward = None
+    if args.backward > 0:
+        s0 = sets[0]
+        g = torch.randn_like(s0["q"])
+        dq, dk, dv = (torch.empty_like(s0["q"]) for _ in range(3))
+        dwk, dwv = torch.empty_like(wk), torch.empty_like(wv)
+        dbias = None if bias is None else torch.empty_like(bias)
+        call = lambda d: sa.slide_attn_backward(ctx, d["q"], d["k"], d["v"], wk, wv, bias, g, dq, dk, dv, dwk, dwv, dbias, stream)
+        for i in range(3):
+            call(sets[i % n_sets])
+        fence()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(args.backward):
+            call(sets[i % n_sets])
+        b.record(stream)
+        fence()
+        assert sa.slide_attn_query_status(ctx) == sa.OK
+        bms = a.elapsed_time(b) / args.backward
+        backward = {"ms_per_step": bms, "steps": args.backward, "value": npx / (bms * 1e-3), "unit": UNIT,
+                    "kernels": "weight transpose, point kernel (a, dl, dq, dW, dbias), gather kernel (dk, dv)"}
+
     # end to end through the host-buffer entry point: pinned host inputs in, pinned result out
     e2e = None
     if args.e2e_steps > 0:
@@ -468,6 +493,8 @@ def main():
             "compute_ceilings": other_rooflines(cfg, main_ms, args.fixed_shift),
             "clocks": clocks, "e2e": e2e,
         }
+        if backward:
+            line["backward"] = backward
         if world == 1 and not args.no_cpu_baseline:
             v, cores, sample = cpu_oracle_rate(cfg, x)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",

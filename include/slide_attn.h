@@ -180,6 +180,32 @@ slide_attn_status slide_attn_detect_fixed_shift(slide_attn_ctx* ctx, const float
 slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* ctx, int* n);
 
 /*
+ * Backward pass of the forward above (training through the module, Sec. 4.3 / Fig. 4 (1); the paper
+ * prints no backward formulas: these are the derivatives of Eq. 2 with the convolution of Eq. 12
+ * inside).  Given dout = d(loss)/d(out), writes the gradients of every input, asynchronously on
+ * `cuda_stream`:
+ *   q, k, v, wk, wv, bias   [in, DEVICE] exactly what the forward was given
+ *   dout                    [in, DEVICE] same shape and dtype as out, 16-byte aligned
+ *   dq, dk, dv              [out, DEVICE] same shape and dtype as q; overwritten
+ *   dwk, dwv                [out, DEVICE] float [C][k*k][k*k]; overwritten (not accumulated into)
+ *   dbias                   [out, DEVICE] float [heads][k*k]; non-NULL iff the context has_bias
+ * For the training-time two-path form (fixed shift + learned kernels, merged weights = their sum)
+ * dwk / dwv ARE the gradients of the learned kernels.  The attention weights are recomputed, so no
+ * forward state is needed.  Supported: head_dim 32, ksize 1 or 3, both dtypes
+ * (SLIDE_ATTN_ERR_UNSUPPORTED otherwise).  Arithmetic is fp32; dq, dk, dv are rounded to the dtype
+ * once; dwk, dwv, dbias are summed over pixels with floating-point atomics, so their last bits may
+ * differ from run to run.  The FIRST backward on a context allocates a scratch buffer of
+ * 2 * B*H*W*heads*k*k floats (cudaMalloc, synchronous); later calls allocate nothing.
+ */
+slide_attn_status slide_attn_backward(slide_attn_ctx* ctx,
+                                      const void* q, const void* k, const void* v,
+                                      const float* wk, const float* wv, const float* bias,
+                                      const void* dout,
+                                      void* dq, void* dk, void* dv,
+                                      float* dwk, float* dwv, float* dbias,
+                                      void* cuda_stream);
+
+/*
  * Waits for `cuda_stream` and reports the device-side status word: SLIDE_ATTN_OK,
  * SLIDE_ATTN_ERR_TIMEOUT if a kernel gave up on a bounded wait, or SLIDE_ATTN_ERR_NOT_FIXED_SHIFT if a
  * forward in fixed-shift mode met a weight that is not one-hot (the output is then undefined).

@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALLOC, ERR_CUDA, ERR_AR
 ERR_TOO_LARGE = 8
 ERR_NOT_FIXED_SHIFT = 9
 
-EXPORTS = ("slide_attn_create", "slide_attn_forward", "slide_attn_forward_host",
+EXPORTS = ("slide_attn_create", "slide_attn_forward", "slide_attn_forward_host", "slide_attn_backward",
            "slide_attn_forward_noalloc",
            "slide_attn_set_variant", "slide_attn_get_variant", "slide_attn_launches_per_forward",
            "slide_attn_set_fixed_shift", "slide_attn_detect_fixed_shift",
@@ -49,6 +49,7 @@ def load() -> ctypes.CDLL:
         lib.slide_attn_create.argtypes = [ctypes.POINTER(vp), i, i, i, i, i, i, i, i]
         lib.slide_attn_forward.argtypes = [vp] * 9
         lib.slide_attn_forward_host.argtypes = [vp] * 9
+        lib.slide_attn_backward.argtypes = [vp] * 15
         lib.slide_attn_forward_noalloc.argtypes = [vp] * 7 + [i] * 7 + [vp]
         lib.slide_attn_set_variant.argtypes = [vp, i]
         lib.slide_attn_get_variant.argtypes = [vp, ctypes.POINTER(i)]
@@ -114,6 +115,13 @@ def slide_attn_forward(ctx, q, k, v, wk, wv, bias, out, stream=None) -> None:
     (default: torch's current stream)."""
     _check(load().slide_attn_forward(ctx, *map(_dev_ptr, (q, k, v, wk, wv, bias, out)),
                                      _stream_ptr(stream)), "slide_attn_forward")
+
+
+def slide_attn_backward(ctx, q, k, v, wk, wv, bias, dout, dq, dk, dv, dwk, dwv, dbias, stream=None) -> None:
+    """Gradients of the forward's inputs for dout = d(loss)/d(out); device tensors, asynchronous on
+    `stream`.  dq, dk, dv: shape and dtype of q; dwk, dwv: float32 like wk; dbias: float32 like bias or None."""
+    _check(load().slide_attn_backward(ctx, *map(_dev_ptr, (q, k, v, wk, wv, bias, dout, dq, dk, dv, dwk, dwv, dbias)),
+                                      _stream_ptr(stream)), "slide_attn_backward")
 
 
 def slide_attn_forward_host(ctx, q, k, v, wk, wv, bias, out, stream=None) -> None:

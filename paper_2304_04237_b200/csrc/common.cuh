@@ -74,6 +74,21 @@ bool shift_supports(int head_dim, int ksize);
 cudaError_t launch_shift_check(const Problem& p, int* d_status, cudaStream_t stream);
 cudaError_t launch_shift(const Problem& p, int* d_status, cudaStream_t stream);
 
+// Backward pass (head_dim 32, k = 1 or 3, both dtypes): gradients of the forward's inputs.
+struct BackwardArgs {
+    const void* dout;    // [B][H][W][heads][head_dim], the problem's dtype
+    void* dq;            // same shape and dtype
+    void* dk;
+    void* dv;
+    float* dwk;          // [C][k*k][k*k]
+    float* dwv;
+    float* dbias;        // [heads][k*k] or nullptr
+};
+bool backward_supports(int head_dim, int ksize);
+size_t backward_workspace_bytes(int B, int H, int W, int heads, int ksize);
+cudaError_t launch_backward(const Problem& p, const BackwardArgs& ga, const void* wt, void* ws, int* d_status,
+                            int num_sms, cudaStream_t stream);
+
 // TILE variant: generic weights, CUDA cores, TMA-staged halo tiles (head_dim 32, k <= 9, both dtypes).
 // Reads the transposed weights that launch_strip_prep writes.
 bool tile_supports(int head_dim, int ksize);

@@ -18,6 +18,7 @@ struct slide_attn_ctx {
     size_t workspace_bytes;
     void* strip_ws;                  // transposed weights of the STRIP variant
     void* umma_ws;                   // bf16 B images of the UMMA_TS variant
+    void* bwd_ws;                    // attention weights and logit gradients between the two backward kernels (first backward)
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
     size_t stage_bytes;
@@ -306,6 +307,44 @@ slide_attn_status slide_attn_forward_host(slide_attn_ctx* c, const void* q, cons
     return SLIDE_ATTN_OK;
 }
 
+slide_attn_status slide_attn_backward(slide_attn_ctx* c, const void* q, const void* k, const void* v,
+                                      const float* wk, const float* wv, const float* bias, const void* dout,
+                                      void* dq, void* dk, void* dv, float* dwk, float* dwv, float* dbias,
+                                      void* cuda_stream)
+{
+    if (!c || !q || !k || !v || !wk || !wv || !dout || !dq || !dk || !dv || !dwk || !dwv) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if ((c->has_bias != 0) != (bias != nullptr) || (c->has_bias != 0) != (dbias != nullptr)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!backward_supports(c->head_dim, c->ksize) || !c->strip_ws) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    const void* ptrs[] = {q, k, v, wk, wv, dout, dq, dk, dv, dwk, dwv};
+    for (const void* p : ptrs) if (!aligned16(p)) return SLIDE_ATTN_ERR_ALIGNMENT;
+    if ((bias && !aligned16(bias)) || (dbias && !aligned16(dbias))) return SLIDE_ATTN_ERR_ALIGNMENT;
+    if (dq == q || dq == k || dq == v || dq == dout || dk == q || dk == k || dk == v || dk == dout ||
+        dv == q || dv == k || dv == v || dv == dout || dq == dk || dq == dv || dk == dv)
+        return SLIDE_ATTN_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!c->bwd_ws) {
+        if (cudaMalloc(&c->bwd_ws, backward_workspace_bytes(c->B, c->H, c->W, c->heads, c->ksize)) != cudaSuccess) {
+            cudaGetLastError();
+            c->bwd_ws = nullptr;
+            return SLIDE_ATTN_ERR_ALLOC;
+        }
+    }
+    Problem p;
+    p.B = c->B; p.H = c->H; p.W = c->W; p.heads = c->heads; p.head_dim = c->head_dim;
+    p.ksize = c->ksize; p.has_bias = c->has_bias; p.dtype = c->dtype;
+    p.q = q; p.k = k; p.v = v; p.wk = wk; p.wv = wv; p.bias = bias; p.out = nullptr;
+    BackwardArgs ga = {dout, dq, dk, dv, dwk, dwv, dbias};
+    const size_t k2 = (size_t)c->ksize * c->ksize;
+    const size_t wbytes = (size_t)c->heads * c->head_dim * k2 * k2 * sizeof(float);
+    bool ok = cudaMemsetAsync(dwk, 0, wbytes, stream) == cudaSuccess && cudaMemsetAsync(dwv, 0, wbytes, stream) == cudaSuccess;
+    if (ok && dbias) ok = cudaMemsetAsync(dbias, 0, (size_t)c->heads * k2 * sizeof(float), stream) == cudaSuccess;
+    if (ok) ok = launch_strip_prep(p, c->strip_ws, stream) == cudaSuccess;
+    if (ok) ok = launch_backward(p, ga, c->strip_ws, c->bwd_ws, c->d_status, c->num_sms, stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+    return SLIDE_ATTN_OK;
+}
+
 slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant variant)
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
@@ -438,6 +477,7 @@ slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
     if (c->workspace) ok &= cudaFree(c->workspace) == cudaSuccess;
     if (c->strip_ws) ok &= cudaFree(c->strip_ws) == cudaSuccess;
     if (c->umma_ws) ok &= cudaFree(c->umma_ws) == cudaSuccess;
+    if (c->bwd_ws) ok &= cudaFree(c->bwd_ws) == cudaSuccess;
     if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
     if (c->host_pipe) {
         ok &= cudaStreamDestroy(c->copy_in) == cudaSuccess;

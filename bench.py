@@ -32,7 +32,7 @@ from paper_2304_04237_b200 import synth  # noqa: E402
 METRIC = "slide_attn_fwd_query_pixels_per_s"
 UNIT = "query-pixels/s"
 FALLBACK_HBM_GBS = 6650.0
-VARIANT_IDS = {"direct": 1, "mma": 2, "umma_ts": 5, "strip": 6, "tile": 8}
+VARIANT_IDS = {"direct": 1, "mma": 2, "umma_ts": 5, "strip": 6, "tile": 8, "mma_wide": 9}
 
 
 def algorithmic_bytes(cfg) -> int:

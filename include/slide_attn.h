@@ -92,11 +92,15 @@ typedef enum {
     SLIDE_ATTN_VARIANT_STRIP   = 6,   /* DIRECT's arithmetic with transposed weights (one coalesced load
                                          per weight) and 4-8 pixels per warp, operands read from global
                                          memory; fp32 FMA; ksize <= 9, any head_dim, fp32 or bf16        */
-    SLIDE_ATTN_VARIANT_TILE    = 8    /* generic weights on the CUDA cores off a TMA-staged halo tile
+    SLIDE_ATTN_VARIANT_TILE    = 8,   /* generic weights on the CUDA cores off a TMA-staged halo tile
                                          in shared memory, 16-byte accesses throughout, convolution
                                          re-associated with the q.k products and the softmax weights;
-                                         head_dim 32, ksize <= 9, fp32 or bf16: what AUTO runs where
-                                         UMMA_TS does not apply                                          */
+                                         head_dim 32, ksize <= 9, fp32 or bf16: what AUTO runs for fp32
+                                         storage                                                         */
+    SLIDE_ATTN_VARIANT_MMA_WIDE = 9   /* large windows with general weights on tensor cores (mma.sync):
+                                         TMA-staged halo tile, weights streamed tap by tap from L2 as
+                                         register fragments; bf16, head_dim 32, ksize 3 / 5 / 7 / 9: what
+                                         AUTO runs for bf16 with ksize >= 5                              */
 } slide_attn_variant;
 
 /*

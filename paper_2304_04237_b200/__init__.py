@@ -3,7 +3,7 @@ C-ABI library in csrc/.  See include/slide_attn.h for the contract."""
 from . import binding  # noqa: F401
 from .binding import (BF16, ERR_ALIGNMENT, ERR_ALLOC, ERR_ARCH, ERR_CUDA, ERR_INVALID_ARG,  # noqa: F401
                       ERR_TIMEOUT, ERR_TOO_LARGE, ERR_NOT_FIXED_SHIFT, ERR_UNSUPPORTED, F32, OK, VARIANT_AUTO, VARIANT_DIRECT,
-                      VARIANT_MMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_TILE, SlideAttnError, slide_attn_create,
+                      VARIANT_MMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_TILE, VARIANT_MMA_WIDE, SlideAttnError, slide_attn_create,
                       slide_attn_destroy, slide_attn_forward, slide_attn_backward, slide_attn_forward_host, slide_attn_forward_noalloc,
                       slide_attn_get_variant, slide_attn_launches_per_forward,
                       slide_attn_profile_begin, slide_attn_profile_end,

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libslide_attn.so")
 
 F32, BF16 = 0, 1
-VARIANT_AUTO, VARIANT_DIRECT, VARIANT_MMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_TILE = 0, 1, 2, 5, 6, 8
+VARIANT_AUTO, VARIANT_DIRECT, VARIANT_MMA, VARIANT_UMMA_TS, VARIANT_STRIP, VARIANT_TILE, VARIANT_MMA_WIDE = 0, 1, 2, 5, 6, 8, 9
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(8)
 ERR_TOO_LARGE = 8
 ERR_NOT_FIXED_SHIFT = 9

@@ -89,6 +89,12 @@ size_t backward_workspace_bytes(int B, int H, int W, int heads, int ksize);
 cudaError_t launch_backward(const Problem& p, const BackwardArgs& ga, const void* wt, void* ws, int* d_status,
                             int num_sms, cudaStream_t stream);
 
+// MMA_WIDE variant: general weights with large windows on mma.sync tensor cores (bf16, head_dim 32,
+// k = 3, 5, 7, 9); a prep launch writes the weights as B fragments into `workspace`.
+bool mma_wide_supports(slide_attn_dtype dtype, int head_dim, int ksize);
+size_t mma_wide_workspace_bytes(int heads, int ksize);
+cudaError_t launch_mma_wide(const Problem& p, void* workspace, int* d_status, cudaStream_t stream);
+
 // TILE variant: generic weights, CUDA cores, TMA-staged halo tiles (head_dim 32, k <= 9, both dtypes).
 // Reads the transposed weights that launch_strip_prep writes.
 bool tile_supports(int head_dim, int ksize);

@@ -18,6 +18,7 @@ struct slide_attn_ctx {
     size_t workspace_bytes;
     void* strip_ws;                  // transposed weights of the STRIP variant
     void* umma_ws;                   // bf16 B images of the UMMA_TS variant
+    void* wide_ws;                   // bf16 B fragments of the MMA_WIDE variant
     void* bwd_ws;                    // attention weights and logit gradients between the two backward kernels (first backward)
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
@@ -55,12 +56,13 @@ bool variant_supported(const slide_attn_ctx* c, slide_attn_variant v) {
         case SLIDE_ATTN_VARIANT_MMA: return c->workspace && mma_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_UMMA_TS: return c->umma_ws && umma_ts_supports(c->dtype, c->head_dim, c->ksize);
         case SLIDE_ATTN_VARIANT_TILE: return c->strip_ws && tile_supports(c->head_dim, c->ksize);
+        case SLIDE_ATTN_VARIANT_MMA_WIDE: return c->wide_ws && mma_wide_supports(c->dtype, c->head_dim, c->ksize);
         default: return false;
     }
 }
 
 slide_attn_variant pick_variant(const slide_attn_ctx* c) {
-    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA_TS, SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_TILE,
+    const slide_attn_variant order[] = {SLIDE_ATTN_VARIANT_UMMA_TS, SLIDE_ATTN_VARIANT_MMA, SLIDE_ATTN_VARIANT_MMA_WIDE, SLIDE_ATTN_VARIANT_TILE,
                                         SLIDE_ATTN_VARIANT_STRIP, SLIDE_ATTN_VARIANT_DIRECT};
     for (slide_attn_variant v : order)
         if (variant_supported(c, v)) return v;
@@ -115,6 +117,10 @@ slide_attn_status launch_problem(slide_attn_ctx* c, const Problem& p, cudaStream
             err = launch_umma_ts_prep(p, c->umma_ws, stream);
             if (ev) cudaEventRecord(ev[1], stream);
             if (err == cudaSuccess) err = launch_umma_ts(p, c->umma_ws, c->d_status, c->num_sms, stream);
+            break;
+        case SLIDE_ATTN_VARIANT_MMA_WIDE:
+            if (ev) cudaEventRecord(ev[1], stream);          // the prep launch is issued inside launch_mma_wide
+            err = launch_mma_wide(p, c->wide_ws, c->d_status, stream);
             break;
         case SLIDE_ATTN_VARIANT_TILE:
             err = launch_strip_prep(p, c->strip_ws, stream);
@@ -190,6 +196,13 @@ slide_attn_status slide_attn_create(slide_attn_ctx** ctx, int B, int H, int W, i
             slide_attn_destroy(c);
             return SLIDE_ATTN_ERR_ALLOC;
         }
+    }
+    if (mma_wide_supports(dtype, head_dim, ksize) &&
+        cudaMalloc(&c->wide_ws, mma_wide_workspace_bytes(heads, ksize)) != cudaSuccess) {
+        cudaGetLastError();
+        c->wide_ws = nullptr;
+        slide_attn_destroy(c);
+        return SLIDE_ATTN_ERR_ALLOC;
     }
     if (strip_supports(head_dim, ksize) &&
         cudaMalloc(&c->strip_ws, strip_workspace_bytes(heads, head_dim, ksize)) != cudaSuccess) {
@@ -350,7 +363,7 @@ slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant v
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
     if (variant == SLIDE_ATTN_VARIANT_AUTO) { c->variant = pick_variant(c); return SLIDE_ATTN_OK; }
     if (variant != SLIDE_ATTN_VARIANT_DIRECT && variant != SLIDE_ATTN_VARIANT_MMA && variant != SLIDE_ATTN_VARIANT_UMMA_TS &&
-        variant != SLIDE_ATTN_VARIANT_STRIP && variant != SLIDE_ATTN_VARIANT_TILE)
+        variant != SLIDE_ATTN_VARIANT_STRIP && variant != SLIDE_ATTN_VARIANT_TILE && variant != SLIDE_ATTN_VARIANT_MMA_WIDE)
         return SLIDE_ATTN_ERR_INVALID_ARG;
     if (!variant_supported(c, variant)) return SLIDE_ATTN_ERR_UNSUPPORTED;
     c->variant = variant;
@@ -405,6 +418,7 @@ slide_attn_status slide_attn_launches_per_forward(const slide_attn_ctx* c, int* 
         case SLIDE_ATTN_VARIANT_STRIP: *n = 2; break;    // weight transpose + fused kernel
         case SLIDE_ATTN_VARIANT_UMMA_TS: *n = 2; break;  // B-image prep + fused kernel
         case SLIDE_ATTN_VARIANT_TILE: *n = 2; break;     // weight transpose + fused kernel
+        case SLIDE_ATTN_VARIANT_MMA_WIDE: *n = 2; break; // weight fragments + fused kernel
         default: *n = 1; break;
     }
     return SLIDE_ATTN_OK;
@@ -478,6 +492,7 @@ slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
     if (c->strip_ws) ok &= cudaFree(c->strip_ws) == cudaSuccess;
     if (c->umma_ws) ok &= cudaFree(c->umma_ws) == cudaSuccess;
     if (c->bwd_ws) ok &= cudaFree(c->bwd_ws) == cudaSuccess;
+    if (c->wide_ws) ok &= cudaFree(c->wide_ws) == cudaSuccess;
     if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
     if (c->host_pipe) {
         ok &= cudaStreamDestroy(c->copy_in) == cudaSuccess;

@@ -15,7 +15,7 @@ from util import TORCH_DTYPE, VARIANTS, assert_close, gpu_forward, to_device
 
 pytestmark = pytest.mark.gpu
 
-ALL_VARIANTS = ["auto", "direct", "strip", "tile", "mma", "umma_ts"]
+ALL_VARIANTS = ["auto", "direct", "strip", "tile", "mma", "mma_wide", "umma_ts"]
 PIPELINED = ["umma_ts"]
 
 
@@ -282,7 +282,7 @@ def test_forward_argument_errors():
         assert lib.slide_attn_forward(ctx, *bad) == sa.ERR_INVALID_ARG
         bad = list(args); bad[1] = args[1] + 4               # misaligned k
         assert lib.slide_attn_forward(ctx, *bad) == sa.ERR_ALIGNMENT
-        assert lib.slide_attn_set_variant(ctx, 9) == sa.ERR_INVALID_ARG
+        assert lib.slide_attn_set_variant(ctx, 10) == sa.ERR_INVALID_ARG and lib.slide_attn_set_variant(ctx, 3) == sa.ERR_INVALID_ARG
         torch.cuda.synchronize()
     finally:
         sa.slide_attn_destroy(ctx)

@@ -8,7 +8,7 @@ import paper_2304_04237_b200 as sa
 TOL = {"f32": 1e-4, "bf16": 2e-2}     # |gpu - ref| <= tol * max(1, |ref|)
 TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
 VARIANTS = {"direct": sa.VARIANT_DIRECT, "mma": sa.VARIANT_MMA, "umma_ts": sa.VARIANT_UMMA_TS, "strip": sa.VARIANT_STRIP,
-            "tile": sa.VARIANT_TILE}
+            "tile": sa.VARIANT_TILE, "mma_wide": sa.VARIANT_MMA_WIDE}
 
 
 def to_device(x, dtype):

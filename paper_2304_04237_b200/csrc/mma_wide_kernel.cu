@@ -21,6 +21,10 @@
 // streams them from L2 tap by tap through a four-stage ring of bulk copies, in the register-fragment
 // order a prep kernel wrote them in: first the k^2 key-side chunks, then the k^2 value-side chunks.
 // Every wait is bounded and sets the status word.
+//
+// Measured and not kept: two M tiles per warp (a weight fragment then feeds two MMAs, but half as many
+// warps with twice the registers ran 1.1-1.9x slower); 16-byte loads of two n-tiles' fragments at once
+// (within +-8 % of the 8-byte form).
 #include "tile_common.cuh"
 
 namespace slide_attn {

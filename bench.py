@@ -309,6 +309,9 @@ def main():
     ap.add_argument("--no-other", action="store_true", help="skip the kernel-only figures of the other gated shapes")
     ap.add_argument("--backward", type=int, default=0, metavar="N",
                     help="also time N backward passes (slide_attn_backward) of the workload and report them beside the forward")
+    ap.add_argument("--block", type=int, default=0, metavar="N",
+                    help="also time N whole blocks (slide_attn_block_forward: Eq. 1 projections, attention, Eq. 3 projection) "
+                         "on the workload's shape and report them beside the forward")
     ap.add_argument("--fixed-shift", action="store_true",
                     help="the workload with exactly one-hot depthwise weights (sigma_w = 0), run in fixed-shift mode")
     args = ap.parse_args()
@@ -435,6 +438,40 @@ def main():
         backward = {"ms_per_step": bms, "steps": args.backward, "value": npx / (bms * 1e-3), "unit": UNIT,
                     "kernels": "weight transpose, point kernel (a, dl, dq, dW, dbias), gather kernel (dk, dv)"}
 
+    # optional: a whole block on the workload's shape (projections on tcgen05 around the attention stage)
+    block = None
+    if args.block > 0 and cfg["dtype"] == "bf16":
+        C = cfg["heads"] * cfg["head_dim"]
+        gen = torch.Generator(device="cuda").manual_seed(1234)
+        xs = [torch.randn((cfg["B"], cfg["H"], cfg["W"], C), device="cuda", generator=gen).to(torch.bfloat16) for _ in range(2)]
+        w_qkv = torch.randn((3, C, C), device="cuda", generator=gen) / C ** 0.5
+        w_o = torch.randn((C, C), device="cuda", generator=gen) / C ** 0.5
+        bout = torch.empty_like(xs[0])
+        ys = [torch.empty_like(xs[0]) for _ in range(3)]
+
+        def timed(fn, n):
+            for i in range(3):
+                fn(i)
+            fence()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(n):
+                fn(i)
+            b.record(stream)
+            fence()
+            assert sa.slide_attn_query_status(ctx) == sa.OK
+            return a.elapsed_time(b) / n
+
+        blk_ms = timed(lambda i: sa.slide_attn_block_forward(ctx, xs[i & 1], w_qkv, w_o, wk, wv, bias, bout, stream), args.block)
+        qkv_ms = timed(lambda i: sa.slide_attn_project(ctx, xs[i & 1], w_qkv, ys, stream), args.block)
+        o_ms = timed(lambda i: sa.slide_attn_project(ctx, xs[i & 1], w_o, [bout], stream), args.block)
+        tok_bytes = npx * C * 2
+        block = {"ms_per_step": blk_ms, "steps": args.block, "value": npx / (blk_ms * 1e-3), "unit": UNIT,
+                 "proj_qkv_ms": qkv_ms, "proj_qkv_gbs": 4 * tok_bytes / (qkv_ms * 1e-3) / 1e9,
+                 "proj_o_ms": o_ms, "proj_o_gbs": 2 * tok_bytes / (o_ms * 1e-3) / 1e9,
+                 "bytes_min_three_stages": 10 * tok_bytes, "bytes_min_fused": 2 * tok_bytes,
+                 "kernels": "weight images + projection GEMM (Eq. 1), attention, weight image + projection GEMM (Eq. 3)"}
+
     # end to end through the host-buffer entry point: pinned host inputs in, pinned result out
     e2e = None
     if args.e2e_steps > 0:
@@ -495,6 +532,8 @@ def main():
         }
         if backward:
             line["backward"] = backward
+        if block:
+            line["block"] = block
         if world == 1 and not args.no_cpu_baseline:
             v, cores, sample = cpu_oracle_rate(cfg, x)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",

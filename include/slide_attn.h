@@ -210,6 +210,39 @@ slide_attn_status slide_attn_backward(slide_attn_ctx* ctx,
                                       void* cuda_stream);
 
 /*
+ * The dense projections around the attention stage (Eq. 1: q = x W_q, k = x W_k, v = x W_v; Eq. 3:
+ * Concat(heads) W_o), as a tensor-core GEMM over the B*H*W tokens of the context's shape:
+ *   y_i[token][o] = sum_c x[token][c] * w[i][c][o],  i = 0 .. nmat-1
+ *   x            [in, DEVICE]  bf16 [B][H][W][C], C = heads*head_dim, 16-byte aligned
+ *   w            [in, DEVICE]  float [nmat][C in][C out], nmat = 1..3 (e.g. W_q, W_k, W_v one after the other)
+ *   y0, y1, y2   [out, DEVICE] bf16 [B][H][W][C] each; the first nmat are written, the rest are ignored
+ * Weights are rounded to bf16, sums are accumulated in fp32, results rounded to bf16 once.  Asynchronous on
+ * `cuda_stream`.  Supported: bf16 contexts with C a multiple of 16, 16 <= C <= 256
+ * (SLIDE_ATTN_ERR_UNSUPPORTED otherwise).  The first call of this function or of slide_attn_block_forward on a
+ * context allocates its scratch (see there); later calls allocate nothing.
+ */
+slide_attn_status slide_attn_project(slide_attn_ctx* ctx, const void* x, const float* w, int nmat,
+                                     void* y0, void* y1, void* y2, void* cuda_stream);
+
+/*
+ * One whole Slide-Attention block (Eq. 1 - 3 with the local attention of Sec. 4 as Eq. 2's attention):
+ *   q, k, v = x W_q, x W_k, x W_v      (Eq. 1; slide_attn_project with nmat = 3)
+ *   z       = slide_attn_forward(q, k, v, wk, wv, bias)     (channel c of q, k, v = head c / head_dim)
+ *   out     = z W_o                    (Eq. 3; slide_attn_project with nmat = 1)
+ *   x, out        [in / out, DEVICE] bf16 [B][H][W][C]; out must not alias x
+ *   w_qkv         [in, DEVICE] float [3][C in][C out]: W_q, W_k, W_v
+ *   w_o           [in, DEVICE] float [C in][C out]
+ *   wk, wv, bias  as in slide_attn_forward
+ * q, k, v and z live in bf16 in a scratch buffer of the context (4 * B*H*W*C*2 bytes plus the bf16 weight
+ * images), allocated with cudaMalloc (synchronous) by the first call; they are rounded to bf16 once each.
+ * The attention stage runs the context's current variant (or the fixed-shift kernel in fixed-shift mode).
+ * Asynchronous on `cuda_stream`; same support as slide_attn_project.
+ */
+slide_attn_status slide_attn_block_forward(slide_attn_ctx* ctx, const void* x, const float* w_qkv,
+                                           const float* w_o, const float* wk, const float* wv,
+                                           const float* bias, void* out, void* cuda_stream);
+
+/*
  * Waits for `cuda_stream` and reports the device-side status word: SLIDE_ATTN_OK,
  * SLIDE_ATTN_ERR_TIMEOUT if a kernel gave up on a bounded wait, or SLIDE_ATTN_ERR_NOT_FIXED_SHIFT if a
  * forward in fixed-shift mode met a weight that is not one-hot (the output is then undefined).

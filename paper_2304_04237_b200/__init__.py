@@ -8,4 +8,5 @@ from .binding import (BF16, ERR_ALIGNMENT, ERR_ALLOC, ERR_ARCH, ERR_CUDA, ERR_IN
                       slide_attn_get_variant, slide_attn_launches_per_forward,
                       slide_attn_profile_begin, slide_attn_profile_end,
                       slide_attn_query_status, slide_attn_set_variant, slide_attn_status_string,
-                      slide_attn_set_fixed_shift, slide_attn_detect_fixed_shift)
+                      slide_attn_set_fixed_shift, slide_attn_detect_fixed_shift,
+                      slide_attn_project, slide_attn_block_forward)

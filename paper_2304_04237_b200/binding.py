@@ -21,7 +21,7 @@ ERR_TOO_LARGE = 8
 ERR_NOT_FIXED_SHIFT = 9
 
 EXPORTS = ("slide_attn_create", "slide_attn_forward", "slide_attn_forward_host", "slide_attn_backward",
-           "slide_attn_forward_noalloc",
+           "slide_attn_forward_noalloc", "slide_attn_project", "slide_attn_block_forward",
            "slide_attn_set_variant", "slide_attn_get_variant", "slide_attn_launches_per_forward",
            "slide_attn_set_fixed_shift", "slide_attn_detect_fixed_shift",
            "slide_attn_profile_begin", "slide_attn_profile_end",
@@ -51,6 +51,8 @@ def load() -> ctypes.CDLL:
         lib.slide_attn_forward_host.argtypes = [vp] * 9
         lib.slide_attn_backward.argtypes = [vp] * 15
         lib.slide_attn_forward_noalloc.argtypes = [vp] * 7 + [i] * 7 + [vp]
+        lib.slide_attn_project.argtypes = [vp, vp, vp, i, vp, vp, vp, vp]
+        lib.slide_attn_block_forward.argtypes = [vp] * 9
         lib.slide_attn_set_variant.argtypes = [vp, i]
         lib.slide_attn_get_variant.argtypes = [vp, ctypes.POINTER(i)]
         lib.slide_attn_set_fixed_shift.argtypes = [vp, i]
@@ -122,6 +124,22 @@ def slide_attn_backward(ctx, q, k, v, wk, wv, bias, dout, dq, dk, dv, dwk, dwv, 
     `stream`.  dq, dk, dv: shape and dtype of q; dwk, dwv: float32 like wk; dbias: float32 like bias or None."""
     _check(load().slide_attn_backward(ctx, *map(_dev_ptr, (q, k, v, wk, wv, bias, dout, dq, dk, dv, dwk, dwv, dbias)),
                                       _stream_ptr(stream)), "slide_attn_backward")
+
+
+def slide_attn_project(ctx, x, w, ys, stream=None) -> None:
+    """Eq. 1 / Eq. 3: ys[i] = x w[i] over the tokens of the context's shape.  x and every ys[i]: bf16 device
+    tensors [B, H, W, C]; w: float32 device tensor [len(ys), C, C] (input channel, output channel)."""
+    ys = list(ys)
+    ptrs = [_dev_ptr(y) for y in ys] + [None] * (3 - len(ys))
+    _check(load().slide_attn_project(ctx, _dev_ptr(x), _dev_ptr(w), len(ys), *ptrs, _stream_ptr(stream)),
+           "slide_attn_project")
+
+
+def slide_attn_block_forward(ctx, x, w_qkv, w_o, wk, wv, bias, out, stream=None) -> None:
+    """A whole block: projections (Eq. 1, w_qkv float32 [3, C, C]), the local attention, output projection
+    (Eq. 3, w_o float32 [C, C]); x and out bf16 device tensors [B, H, W, C]."""
+    _check(load().slide_attn_block_forward(ctx, *map(_dev_ptr, (x, w_qkv, w_o, wk, wv, bias, out)),
+                                           _stream_ptr(stream)), "slide_attn_block_forward")
 
 
 def slide_attn_forward_host(ctx, q, k, v, wk, wv, bias, out, stream=None) -> None:

@@ -20,6 +20,7 @@ struct slide_attn_ctx {
     void* umma_ws;                   // bf16 B images of the UMMA_TS variant
     void* wide_ws;                   // bf16 B fragments of the MMA_WIDE variant
     void* bwd_ws;                    // attention weights and logit gradients between the two backward kernels (first backward)
+    void* block_ws;                  // q, k, v, z of slide_attn_block_forward and the projections' weight images (first use)
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
     size_t stage_bytes;
@@ -358,6 +359,96 @@ slide_attn_status slide_attn_backward(slide_attn_ctx* c, const void* q, const vo
     return SLIDE_ATTN_OK;
 }
 
+namespace {
+
+size_t block_tensor_bytes(const slide_attn_ctx* c) {
+    const size_t raw = (size_t)c->B * c->H * c->W * c->heads * c->head_dim * 2;
+    return (raw + 255) & ~(size_t)255;
+}
+
+// Scratch of the projections: four bf16 token tensors, then the weight images of Eq. 1 and of Eq. 3.
+slide_attn_status block_scratch(slide_attn_ctx* c) {
+    const int C = c->heads * c->head_dim;
+    if (c->dtype != SLIDE_ATTN_BF16 || !proj_supports(C, C)) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    if ((long long)c->B * c->H * c->W > 0x7fffff00LL) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    if (c->block_ws) return SLIDE_ATTN_OK;
+    if (proj_setup() != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+    const size_t total = 4 * block_tensor_bytes(c) + proj_workspace_bytes(C, C, 3) + proj_workspace_bytes(C, C, 1);
+    if (cudaMalloc(&c->block_ws, total) != cudaSuccess) {
+        cudaGetLastError();
+        c->block_ws = nullptr;
+        return SLIDE_ATTN_ERR_ALLOC;
+    }
+    return SLIDE_ATTN_OK;
+}
+
+}  // namespace
+
+slide_attn_status slide_attn_project(slide_attn_ctx* c, const void* x, const float* w, int nmat,
+                                     void* y0, void* y1, void* y2, void* cuda_stream)
+{
+    if (!c || !x || !w || nmat < 1 || nmat > 3 || !y0 || (nmat > 1 && !y1) || (nmat > 2 && !y2)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    void* y[3] = {y0, nmat > 1 ? y1 : nullptr, nmat > 2 ? y2 : nullptr};
+    if (!aligned16(x) || !aligned16(w)) return SLIDE_ATTN_ERR_ALIGNMENT;
+    for (int i = 0; i < nmat; ++i) {
+        if (!aligned16(y[i])) return SLIDE_ATTN_ERR_ALIGNMENT;
+        if (y[i] == x) return SLIDE_ATTN_ERR_INVALID_ARG;
+        for (int j = 0; j < i; ++j) if (y[i] == y[j]) return SLIDE_ATTN_ERR_INVALID_ARG;
+    }
+    slide_attn_status st = block_scratch(c);
+    if (st != SLIDE_ATTN_OK) return st;
+    const int C = c->heads * c->head_dim;
+    unsigned char* img = static_cast<unsigned char*>(c->block_ws) + 4 * block_tensor_bytes(c);
+    if (launch_proj(x, (long long)c->B * c->H * c->W, C, w, C, nmat, y, img, c->d_status, c->num_sms,
+                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    return SLIDE_ATTN_OK;
+}
+
+slide_attn_status slide_attn_block_forward(slide_attn_ctx* c, const void* x, const float* w_qkv, const float* w_o,
+                                           const float* wk, const float* wv, const float* bias, void* out,
+                                           void* cuda_stream)
+{
+    if (!c || !x || !w_qkv || !w_o || !wk || !wv || !out) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if ((c->has_bias != 0) != (bias != nullptr)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (out == x) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!on_ctx_device(c)) return SLIDE_ATTN_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(out) || !aligned16(w_qkv) || !aligned16(w_o) || !aligned16(wk) || !aligned16(wv) ||
+        (bias && !aligned16(bias)))
+        return SLIDE_ATTN_ERR_ALIGNMENT;
+    slide_attn_status st = block_scratch(c);
+    if (st != SLIDE_ATTN_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int C = c->heads * c->head_dim;
+    const long long rows = (long long)c->B * c->H * c->W;
+    const size_t tb = block_tensor_bytes(c);
+    unsigned char* base = static_cast<unsigned char*>(c->block_ws);
+    void* qkv[3] = {base, base + tb, base + 2 * tb};
+    void* z = base + 3 * tb;
+    unsigned char* img_qkv = base + 4 * tb;
+    unsigned char* img_o = img_qkv + proj_workspace_bytes(C, C, 3);
+
+    if (launch_proj(x, rows, C, w_qkv, C, 3, qkv, img_qkv, c->d_status, c->num_sms, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    Problem p;
+    p.B = c->B; p.H = c->H; p.W = c->W; p.heads = c->heads; p.head_dim = c->head_dim;
+    p.ksize = c->ksize; p.has_bias = c->has_bias; p.dtype = c->dtype;
+    p.q = qkv[0]; p.k = qkv[1]; p.v = qkv[2]; p.wk = wk; p.wv = wv; p.bias = bias; p.out = z;
+    st = launch_problem(c, p, stream, false);
+    if (st != SLIDE_ATTN_OK) return st;
+    void* ys[1] = {out};
+    if (launch_proj(z, rows, C, w_o, C, 1, ys, img_o, c->d_status, c->num_sms, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SLIDE_ATTN_ERR_CUDA;
+    }
+    return SLIDE_ATTN_OK;
+}
+
 slide_attn_status slide_attn_set_variant(slide_attn_ctx* c, slide_attn_variant variant)
 {
     if (!c) return SLIDE_ATTN_ERR_INVALID_ARG;
@@ -493,6 +584,7 @@ slide_attn_status slide_attn_destroy(slide_attn_ctx* c)
     if (c->umma_ws) ok &= cudaFree(c->umma_ws) == cudaSuccess;
     if (c->bwd_ws) ok &= cudaFree(c->bwd_ws) == cudaSuccess;
     if (c->wide_ws) ok &= cudaFree(c->wide_ws) == cudaSuccess;
+    if (c->block_ws) ok &= cudaFree(c->block_ws) == cudaSuccess;
     if (c->stage) ok &= cudaFree(c->stage) == cudaSuccess;
     if (c->host_pipe) {
         ok &= cudaStreamDestroy(c->copy_in) == cudaSuccess;

@@ -218,8 +218,8 @@ slide_attn_status slide_attn_backward(slide_attn_ctx* ctx,
  *   y0, y1, y2   [out, DEVICE] bf16 [B][H][W][C] each; the first nmat are written, the rest are ignored
  * Weights are rounded to bf16, sums are accumulated in fp32, results rounded to bf16 once.  Asynchronous on
  * `cuda_stream`.  Supported: bf16 contexts with C a multiple of 16, 16 <= C <= 256
- * (SLIDE_ATTN_ERR_UNSUPPORTED otherwise).  The first call of this function or of slide_attn_block_forward on a
- * context allocates its scratch (see there); later calls allocate nothing.
+ * (SLIDE_ATTN_ERR_UNSUPPORTED otherwise).  Allocates nothing; one kernel launch (two to twelve when C > 128, where
+ * the weights of all output columns do not fit shared memory together).
  */
 slide_attn_status slide_attn_project(slide_attn_ctx* ctx, const void* x, const float* w, int nmat,
                                      void* y0, void* y1, void* y2, void* cuda_stream);
@@ -233,8 +233,8 @@ slide_attn_status slide_attn_project(slide_attn_ctx* ctx, const void* x, const f
  *   w_qkv         [in, DEVICE] float [3][C in][C out]: W_q, W_k, W_v
  *   w_o           [in, DEVICE] float [C in][C out]
  *   wk, wv, bias  as in slide_attn_forward
- * q, k, v and z live in bf16 in a scratch buffer of the context (4 * B*H*W*C*2 bytes plus the bf16 weight
- * images), allocated with cudaMalloc (synchronous) by the first call; they are rounded to bf16 once each.
+ * q, k, v and z live in bf16 in a scratch buffer of the context (4 * B*H*W*C*2 bytes), allocated with
+ * cudaMalloc (synchronous) by the first call; they are rounded to bf16 once each.
  * The attention stage runs the context's current variant (or the fixed-shift kernel in fixed-shift mode).
  * Asynchronous on `cuda_stream`; same support as slide_attn_project.
  */

@@ -101,12 +101,10 @@ bool tile_supports(int head_dim, int ksize);
 cudaError_t launch_tile(const Problem& p, const void* workspace, int* d_status, cudaStream_t stream);
 
 // Projections of a block (Eq. 1 / Eq. 3) as a tcgen05 GEMM: y[i] = x w[i] for nmat row-major fp32 [c_in][c_out]
-// matrices, x and y bf16 with channels contiguous.  `workspace` receives the bf16 weight images
-// (proj_workspace_bytes); proj_setup must have succeeded once on the device.
+// matrices, x and y bf16 with channels contiguous.  proj_setup must have succeeded once on the device.
 bool proj_supports(int c_in, int c_out);
-size_t proj_workspace_bytes(int c_in, int c_out, int nmat);
 cudaError_t proj_setup();
 cudaError_t launch_proj(const void* x, long long rows, int c_in, const float* w, int c_out, int nmat,
-                        void* const* y, void* workspace, int* d_status, int num_sms, cudaStream_t stream);
+                        void* const* y, int* d_status, int num_sms, cudaStream_t stream);
 
 }  // namespace slide_attn

@@ -1,6 +1,8 @@
 // Projections of a Slide-Attention block (Eq. 1: q = x W_q, k = x W_k, v = x W_v; Eq. 3: Concat(heads) W_o)
 // as one persistent tcgen05 GEMM:  Y[rows x N] = X[rows x K] W[K x N], X and Y bf16 (token-major, channels
-// contiguous), W given in fp32 and rounded to bf16 once by a prep launch, fp32 accumulation in tensor memory.
+// contiguous), W given in fp32 and rounded to bf16 once as each CTA lays it out in its shared memory, fp32
+// accumulation in tensor memory.  One launch per projection call (several when the weights of all output columns
+// do not fit shared memory together).
 //
 // The column range of one launch is split into chunks of `nch` columns (one MMA shape); all chunk images of the
 // launch stay resident in shared memory, X comes in as 128-row tiles through a TMA ring.  K <= 256 is one tile
@@ -8,10 +10,11 @@
 //
 // Shared-memory operand layout (no swizzle, K-major core matrices of 8 rows x 16 bytes):
 //   X tile   [K/8][128 rows][16 B]   written by K/8 TMA boxes of 8 channels x 128 rows (rows past the end read 0)
-//   W chunk  [K/8][nch cols][16 B]   written by the prep kernel, copied in with one bulk copy per launch
+//   W chunk  [K/8][nch cols][16 B]   built from the fp32 weights by the epilogue warps while the first X tiles load
 //
-// Warps: 0 TMA producer, 1 MMA issuer (owns tensor memory), 2-5 epilogue (TMEM lane quarter = warp % 4: one
-// thread per output row, tcgen05.ld.32x32b -> bf16 -> 16-byte stores).  Two accumulator slots of 256 columns let
+// Warps: 0 TMA producer, 1 MMA issuer (owns tensor memory), 2-9 epilogue (TMEM lane quarter = warp % 4, two warps
+// per quarter taking the column passes in turn: one thread per accumulator row, tcgen05.ld.32x32b -> bf16 -> a padded staging patch in shared memory -> row-major
+// 16-byte stores of whole sectors).  Two accumulator slots of 256 columns let
 // the MMAs of item i+1 run under the epilogue of item i.  Every wait is bounded; a wait that runs out sets the
 // status word and the kernel still releases tensor memory.
 #include "common.cuh"
@@ -21,64 +24,74 @@ namespace slide_attn {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter: they take the column passes of an item in turn
+constexpr int kThreads = (2 + kEpiWarps) * 32;
 constexpr int kMaxStages = 6;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = 256;
 constexpr size_t kMaxSmem = 227 * 1024;
-constexpr size_t kMaxImage = 96 * 1024;      // resident weight chunks of one launch
 
 constexpr int kBarXFull = 0;                 // [kMaxStages]
 constexpr int kBarXEmpty = kMaxStages;       // [kMaxStages]  one arrival: the commit behind the tile's last MMA
-constexpr int kBarWeights = 2 * kMaxStages;
+constexpr int kBarWeights = 2 * kMaxStages;  // count kEpiWarps: the weight images are in shared memory
 constexpr int kBarAccFull = kBarWeights + 1; // [2]
-constexpr int kBarAccFree = kBarAccFull + 2; // [2]  count 4 (epilogue warps)
+constexpr int kBarAccFree = kBarAccFull + 2; // [2]  count kEpiWarps
 constexpr int kNumBars = kBarAccFree + 2;
 
 struct ProjParams {
-    const unsigned char* img;    // chunk images of this launch, chunk after chunk
+    const float* w;              // nmat row-major [K][ycols] matrices, one after the other
     __nv_bfloat16* y[3];         // output tensors, each [rows][ycols]
-    int ycols;                   // channels of one output tensor
+    int ycols;                   // channels of one output tensor = columns of one weight matrix
     int n0;                      // first column of this launch, counted over the concatenated output tensors
     int rows, K, nch, nchunks, stages;
+    int sw_max;                  // widest epilogue pass in columns: 64 or 32 (sizes the staging patches)
     int* status;
 };
 
-__device__ __forceinline__ void tmem_ld_32x32b_x16_wait(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr) : "memory");
+
+// One epilogue pass of a warp: SW accumulator columns of its 32 rows -> bf16 -> global memory (see the kernel).
+template <int SW>
+__device__ __forceinline__ void store_cols(uint32_t taddr, unsigned char* stg, int lane, __nv_bfloat16* ybase, int ycols,
+                                           int rows_left)
+{
+    constexpr int RS = SW * 2 + 16;
+    uint32_t r[SW];
+    // all loads of the pass are in flight before the one wait
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int c = 0; c < SW; c += 16)
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(r[c + 0]), "=r"(r[c + 1]), "=r"(r[c + 2]), "=r"(r[c + 3]), "=r"(r[c + 4]), "=r"(r[c + 5]), "=r"(r[c + 6]),
+              "=r"(r[c + 7]), "=r"(r[c + 8]), "=r"(r[c + 9]), "=r"(r[c + 10]), "=r"(r[c + 11]), "=r"(r[c + 12]), "=r"(r[c + 13]),
+              "=r"(r[c + 14]), "=r"(r[c + 15])
+            : "r"(taddr + (uint32_t)c) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int c = 0; c < SW; c += 8) {
+        // the registers are passed through an empty asm so that no use of them is scheduled above the wait
+        asm volatile("" : "+r"(r[c]), "+r"(r[c + 1]), "+r"(r[c + 2]), "+r"(r[c + 3]), "+r"(r[c + 4]), "+r"(r[c + 5]), "+r"(r[c + 6]), "+r"(r[c + 7]));
+        *reinterpret_cast<uint4*>(stg + lane * RS + c * 2) =
+            make_uint4(pack_bf16(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), pack_bf16(__uint_as_float(r[c + 2]), __uint_as_float(r[c + 3])),
+                       pack_bf16(__uint_as_float(r[c + 4]), __uint_as_float(r[c + 5])), pack_bf16(__uint_as_float(r[c + 6]), __uint_as_float(r[c + 7])));
+    }
+    __syncwarp();
+    constexpr int PR = SW / 8;                            // 16-byte pieces per row
+    uint4 piece[PR];
+#pragma unroll
+    for (int j = 0; j < PR; ++j) {
+        const int p = j * 32 + lane;
+        piece[j] = *reinterpret_cast<const uint4*>(stg + (p / PR) * RS + (p % PR) * 16);
+    }
+#pragma unroll
+    for (int j = 0; j < PR; ++j) {
+        const int p = j * 32 + lane, rr = p / PR, pc = p % PR;
+        if (rr < rows_left) *reinterpret_cast<uint4*>(ybase + (size_t)rr * ycols + pc * 8) = piece[j];
+    }
+    __syncwarp();
 }
 
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity) ? 1 : 0) != 0;
-}
-
-// bf16 images of the weights, one per chunk of nch columns: [chunk][K/8][nch][8 K-consecutive bf16].
-// `w` holds `nmat` row-major [K][ncols] fp32 matrices one after the other; output column n of the concatenation
-// is column n % ncols of matrix n / ncols.
-__global__ void __launch_bounds__(256)
-proj_prep_kernel(const float* __restrict__ w, int K, int ncols, int nmat, int nch, unsigned char* __restrict__ img)
-{
-    grid_launch_dependents();
-    const int ntot = ncols * nmat, kgs = K >> 3;
-    const size_t chunk_bytes = (size_t)kgs * nch * 16;
-    for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < kgs * ntot; item += gridDim.x * blockDim.x) {
-        const int kg = item / ntot, n = item - kg * ntot;
-        const float* src = w + (size_t)(n / ncols) * K * ncols + (size_t)(8 * kg) * ncols + (n % ncols);
-        float val[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) val[e] = src[(size_t)e * ncols];
-        unsigned char* dst = img + (size_t)(n / nch) * chunk_bytes + ((size_t)kg * nch + (n % nch)) * 16;
-        *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(val[0], val[1]), pack_bf16(val[2], val[3]),
-                                                    pack_bf16(val[4], val[5]), pack_bf16(val[6], val[7]));
-    }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -92,6 +105,7 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
     const uint32_t x_off = img_pad;
     const uint32_t tmem_off = x_off + (uint32_t)P.stages * stage_bytes;
     const uint32_t bar0 = smem_u32(smem + tmem_off + 16);
+    const uint32_t stage_off = (tmem_off + 16 + 16 + kNumBars * 8 + 15u) & ~15u;   // epilogue staging, 16-byte aligned
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
@@ -101,8 +115,8 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init_only(bar(kBarXFull + s), 1); mbar_init_only(bar(kBarXEmpty + s), 1); }
-        mbar_init_only(bar(kBarWeights), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init_only(bar(kBarAccFull + i), 1); mbar_init_only(bar(kBarAccFree + i), 4); }
+        mbar_init_only(bar(kBarWeights), kEpiWarps);
+        for (int i = 0; i < 2; ++i) { mbar_init_only(bar(kBarAccFull + i), 1); mbar_init_only(bar(kBarAccFree + i), kEpiWarps); }
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(smem + tmem_off), kTmemCols);
@@ -113,14 +127,11 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
     bool ok = true;
 
     if (warp == 0) {
-        // ---- TMA producer: the weight images once, then the X tiles of this CTA through the ring.  Everything
-        // this kernel reads from global memory is read here, after the kernels ahead of it in the stream have
-        // completed (the kernel may have been launched before they did).
+        // ---- TMA producer: the X tiles of this CTA through the ring.  The kernel may have been launched before the
+        // kernels ahead of it in the stream completed, so every thread that reads global memory waits for them first.
         uint32_t leader;
         if (elect_one(leader) && my_tiles > 0) {
             grid_dependency_wait();
-            mbar_expect_tx(bar(kBarWeights), img_bytes);
-            bulk_load_1d(smem_u32(smem), P.img, img_bytes, bar(kBarWeights));
             for (int t = 0; ok && t < my_tiles; ++t) {
                 const int s = t % S, m = (int)blockIdx.x + t * (int)gridDim.x;
                 if (!mbar_wait(bar(kBarXEmpty + s), (uint32_t)(((t / S) & 1) ^ 1))) { ok = false; break; }
@@ -160,27 +171,54 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
     } else {
-        // ---- epilogue: thread = output row 32 (warp % 4) + lane of the tile
-        const int sub = warp & 3;
+        // ---- epilogue: lane = accumulator row 32 (warp % 4) + lane of the tile.  Each pass takes up to 64 columns:
+        // the lane's row goes TMEM -> registers -> bf16 -> a staging row of this warp in shared memory (row pitch
+        // 2 SW + 16 bytes: conflict-free 16-byte stores), then the warp writes the 32 x SW patch to global memory in
+        // row-major order, 16 bytes per lane, so that every row segment leaves as whole 32-byte sectors.
+        const int sub = warp & 3, half = (warp - 2) >> 2;
         const uint32_t tlane = tmem + ((uint32_t)(32 * sub) << 16);
+        unsigned char* stg = smem + stage_off + (size_t)(warp - 2) * (size_t)(32 * (P.sw_max * 2 + 16));
+        if (my_tiles > 0) {
+            // the bf16 weight images of this launch's columns: [chunk][K/8][nch][8 K-consecutive bf16]; consecutive
+            // threads take consecutive columns, so the fp32 reads are coalesced
+            grid_dependency_wait();
+            const int ncl = P.nchunks * P.nch, kgs = P.K >> 3;
+            const uint32_t chunk_bytes = (uint32_t)kgs * (uint32_t)P.nch * 16u;
+            for (int item = (int)threadIdx.x - 64; item < kgs * ncl; item += kEpiWarps * 32) {
+                const int kg = item / ncl, nl = item - kg * ncl;
+                const int n = P.n0 + nl, mat = n / P.ycols, col = n - mat * P.ycols;
+                const float* src = P.w + ((size_t)mat * P.K + 8 * kg) * P.ycols + col;
+                float val[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) val[e] = src[(size_t)e * P.ycols];
+                const int chn = nl / P.nch;
+                *reinterpret_cast<uint4*>(smem + (size_t)chn * chunk_bytes + ((size_t)kg * P.nch + (nl - chn * P.nch)) * 16) =
+                    make_uint4(pack_bf16(val[0], val[1]), pack_bf16(val[2], val[3]), pack_bf16(val[4], val[5]), pack_bf16(val[6], val[7]));
+            }
+            fence_proxy_async_smem();            // the tensor core reads these bytes through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarWeights));
+        }
         int it = 0;
         for (int t = 0; ok && t < my_tiles; ++t) {
-            const long long row = ((long long)blockIdx.x + (long long)t * gridDim.x) * 128 + 32 * sub + lane;
-            const bool live = row < (long long)P.rows;
+            const long long row0 = ((long long)blockIdx.x + (long long)t * gridDim.x) * 128 + 32 * sub;
+            const int rows_left = (long long)P.rows - row0 > 32 ? 32 : (int)((long long)P.rows - row0);   // may be <= 0
             for (int ch = 0; ch < P.nchunks; ++ch, ++it) {
                 const int slot = it & 1;
                 if (!warp_wait(bar(kBarAccFull + slot), (uint32_t)((it >> 1) & 1))) { ok = false; break; }
                 tc_fence_after_sync();
-                for (int c = 0; c < P.nch; c += 16) {
-                    float a[16];
-                    tmem_ld_32x32b_x16_wait(tlane + (uint32_t)slot * kSlotCols + (uint32_t)c, a);
-                    const int n = P.n0 + ch * P.nch + c;                 // 16 columns never straddle two tensors
+                const uint32_t tacc = tlane + (uint32_t)slot * kSlotCols;
+                int c = 0;
+                for (int pass = 0; c < P.nch; ++pass) {
+                    const int sw = (P.nch - c >= 64 && P.sw_max >= 64) ? 64 : (P.nch - c >= 32 ? 32 : 16);
+                    if (((pass + it) & 1) != half) { c += sw; continue; }
+                    const int n = P.n0 + ch * P.nch + c;                 // a pass never straddles two tensors
                     const int ti = n / P.ycols, col = n - ti * P.ycols;
-                    if (live) {
-                        uint4* dst = reinterpret_cast<uint4*>(P.y[ti] + (size_t)row * P.ycols + col);
-                        dst[0] = make_uint4(pack_bf16(a[0], a[1]), pack_bf16(a[2], a[3]), pack_bf16(a[4], a[5]), pack_bf16(a[6], a[7]));
-                        dst[1] = make_uint4(pack_bf16(a[8], a[9]), pack_bf16(a[10], a[11]), pack_bf16(a[12], a[13]), pack_bf16(a[14], a[15]));
-                    }
+                    __nv_bfloat16* ybase = P.y[ti] + (size_t)row0 * P.ycols + col;
+                    if (sw == 64) store_cols<64>(tacc + (uint32_t)c, stg, lane, ybase, P.ycols, rows_left);
+                    else if (sw == 32) store_cols<32>(tacc + (uint32_t)c, stg, lane, ybase, P.ycols, rows_left);
+                    else store_cols<16>(tacc + (uint32_t)c, stg, lane, ybase, P.ycols, rows_left);
+                    c += sw;
                 }
                 tc_fence_before_sync();
                 __syncwarp();
@@ -195,24 +233,49 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-size_t smem_bytes(int K, int nch, int nchunks, int stages) {
+size_t smem_bytes(int K, int nch, int nchunks, int stages, int sw_max) {
     const size_t img = ((size_t)nchunks * (K / 8) * nch * 16 + 127) & ~(size_t)127;
-    return img + (size_t)stages * K * 256 + 16 + 16 + kNumBars * 8 + 128;
+    return img + (size_t)stages * K * 256 + 16 + 16 + kNumBars * 8 + 16 + (size_t)kEpiWarps * 32 * (sw_max * 2 + 16) + 128;
+}
+
+// Columns per chunk (one MMA shape: a multiple of 16, at most 256, dividing the columns of one tensor), chunks per
+// launch, X stages (at least two) and the widest epilogue pass, such that everything fits shared memory.  Fewest
+// launches win (every launch reads X again).
+struct Plan { int nch, per_launch, stages, sw_max; };
+
+bool make_plan(int c_in, int c_out, int nmat, Plan* plan) {
+    bool found = false;
+    long best_score = 0;
+    for (int div = 1; div <= 16; ++div) {
+        if (c_out % div != 0) continue;
+        const int nch = c_out / div;
+        if (nch > 256 || nch % 16 != 0) continue;
+        const int total = (c_out / nch) * nmat;
+        for (int sw = 64; sw >= 32; sw -= 32) {
+            for (int stages = kMaxStages; stages >= 2; --stages) {
+                int per = total;
+                while (per >= 1 && smem_bytes(c_in, nch, per, stages, sw) > kMaxSmem) --per;
+                if (per < 1) continue;
+                const int launches = (total + per - 1) / per;
+                // fewest launches; then up to four stages; then the wide pass; then more stages; then the wide chunk
+                const long score = -(long)launches * 1000000 + (stages < 4 ? stages : 4) * 10000 + sw * 100 + stages * 10 + (nch > 128 ? 2 : nch > 64 ? 1 : 0);
+                if (!found || score > best_score) {
+                    found = true; best_score = score;
+                    plan->nch = nch; plan->per_launch = per; plan->stages = stages; plan->sw_max = sw;
+                }
+            }
+        }
+    }
+    return found;
 }
 
 }  // namespace
 
 bool proj_supports(int c_in, int c_out) {
-    return c_in >= 16 && c_in <= 256 && c_in % 16 == 0 && c_out >= 16 && c_out <= 256 && c_out % 16 == 0;
+    Plan pl;
+    return c_in >= 16 && c_in <= 256 && c_in % 16 == 0 && c_out >= 16 && c_out <= 256 && c_out % 16 == 0 &&
+           make_plan(c_in, c_out, 1, &pl);
 }
-
-// columns per chunk: the whole tensor when its image fits the resident budget, else half of it
-static int chunk_cols(int c_in, int c_out) {
-    if ((size_t)c_in * c_out * 2 <= kMaxImage) return c_out;
-    return (c_out / 2) % 16 == 0 ? c_out / 2 : 0;
-}
-
-size_t proj_workspace_bytes(int c_in, int c_out, int nmat) { return (size_t)c_in * c_out * nmat * 2; }
 
 cudaError_t proj_setup() {
     if (!tensor_map_available()) return cudaErrorNotSupported;
@@ -220,51 +283,37 @@ cudaError_t proj_setup() {
 }
 
 cudaError_t launch_proj(const void* x, long long rows, int c_in, const float* w, int c_out, int nmat,
-                        void* const* y, void* workspace, int* d_status, int num_sms, cudaStream_t stream)
+                        void* const* y, int* d_status, int num_sms, cudaStream_t stream)
 {
-    if (!proj_supports(c_in, c_out) || nmat < 1 || nmat > 3 || rows < 1 || rows > 0x7fffff00LL) return cudaErrorInvalidValue;
-    const int nch = chunk_cols(c_in, c_out);
-    if (nch == 0) return cudaErrorInvalidValue;
-    unsigned char* img = static_cast<unsigned char*>(workspace);
-    const int ntot = c_out * nmat;
-    {
-        const int items = (c_in / 8) * ntot;
-        proj_prep_kernel<<<(items + 255) / 256, 256, 0, stream>>>(w, c_in, c_out, nmat, nch, img);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
+    Plan pl;
+    if (!proj_supports(c_in, c_out) || nmat < 1 || nmat > 3 || rows < 1 || rows > 0x7fffff00LL ||
+        !make_plan(c_in, c_out, nmat, &pl))
+        return cudaErrorInvalidValue;
     CUtensorMap map_x;
     if (!make_tile_map(&map_x, x, 2, 1, 1, (int)rows, c_in, 8, 128, 1)) return cudaErrorInvalidValue;
 
-    const size_t chunk_bytes = (size_t)(c_in / 8) * nch * 16;
-    const int total_chunks = ntot / nch;
-    int per_launch = (int)(kMaxImage / chunk_bytes);
-    if (per_launch < 1) return cudaErrorInvalidValue;
-    if (per_launch > total_chunks) per_launch = total_chunks;
+    const int total_chunks = (c_out / pl.nch) * nmat;
     const int ntiles = (int)((rows + 127) / 128);
-    bool first = true;
-    for (int c0 = 0; c0 < total_chunks; c0 += per_launch) {
-        const int nchunks = total_chunks - c0 < per_launch ? total_chunks - c0 : per_launch;
-        int stages = kMaxStages;
-        while (stages >= 2 && smem_bytes(c_in, nch, nchunks, stages) > kMaxSmem) --stages;
-        if (stages < 2) return cudaErrorInvalidConfiguration;
+    for (int c0 = 0; c0 < total_chunks; c0 += pl.per_launch) {
+        const int nchunks = total_chunks - c0 < pl.per_launch ? total_chunks - c0 : pl.per_launch;
         ProjParams P;
-        P.img = img + (size_t)c0 * chunk_bytes;
+        P.w = w;
         for (int i = 0; i < 3; ++i) P.y[i] = static_cast<__nv_bfloat16*>(i < nmat ? y[i] : nullptr);
-        P.ycols = c_out; P.n0 = c0 * nch;
-        P.rows = (int)rows; P.K = c_in; P.nch = nch; P.nchunks = nchunks; P.stages = stages;
+        P.ycols = c_out; P.n0 = c0 * pl.nch;
+        P.rows = (int)rows; P.K = c_in; P.nch = pl.nch; P.nchunks = nchunks; P.stages = pl.stages; P.sw_max = pl.sw_max;
         P.status = d_status;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(ntiles < num_sms ? ntiles : num_sms));
         cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = smem_bytes(c_in, nch, nchunks, stages);
+        cfg.dynamicSmemBytes = smem_bytes(c_in, pl.nch, nchunks, pl.stages, pl.sw_max);
         cfg.stream = stream;
+        // the launch may begin (barriers, tensor memory) while the kernel ahead of it in the stream drains; every
+        // thread that reads global memory waits for that kernel first
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = first ? 1 : 0;          // only the launch right behind the prep kernel overlaps it
-        first = false;
+        cfg.numAttrs = 1;
         cudaError_t e = cudaLaunchKernelEx(&cfg, proj_kernel, map_x, P);
         if (e != cudaSuccess) return e;
     }

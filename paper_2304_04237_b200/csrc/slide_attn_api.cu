@@ -20,7 +20,8 @@ struct slide_attn_ctx {
     void* umma_ws;                   // bf16 B images of the UMMA_TS variant
     void* wide_ws;                   // bf16 B fragments of the MMA_WIDE variant
     void* bwd_ws;                    // attention weights and logit gradients between the two backward kernels (first backward)
-    void* block_ws;                  // q, k, v, z of slide_attn_block_forward and the projections' weight images (first use)
+    void* block_ws;                  // q, k, v, z of slide_attn_block_forward (first use)
+    bool proj_ready;                 // the projection kernel's attributes are set on this device
     // staging buffers for slide_attn_forward_host, allocated on first use
     void* stage;
     size_t stage_bytes;
@@ -366,14 +367,23 @@ size_t block_tensor_bytes(const slide_attn_ctx* c) {
     return (raw + 255) & ~(size_t)255;
 }
 
-// Scratch of the projections: four bf16 token tensors, then the weight images of Eq. 1 and of Eq. 3.
-slide_attn_status block_scratch(slide_attn_ctx* c) {
+slide_attn_status proj_check(slide_attn_ctx* c) {
     const int C = c->heads * c->head_dim;
     if (c->dtype != SLIDE_ATTN_BF16 || !proj_supports(C, C)) return SLIDE_ATTN_ERR_UNSUPPORTED;
     if ((long long)c->B * c->H * c->W > 0x7fffff00LL) return SLIDE_ATTN_ERR_UNSUPPORTED;
+    if (!c->proj_ready) {
+        if (proj_setup() != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
+        c->proj_ready = true;
+    }
+    return SLIDE_ATTN_OK;
+}
+
+// Scratch of the block: four bf16 token tensors (q, k, v, z).
+slide_attn_status block_scratch(slide_attn_ctx* c) {
+    slide_attn_status st = proj_check(c);
+    if (st != SLIDE_ATTN_OK) return st;
     if (c->block_ws) return SLIDE_ATTN_OK;
-    if (proj_setup() != cudaSuccess) { cudaGetLastError(); return SLIDE_ATTN_ERR_CUDA; }
-    const size_t total = 4 * block_tensor_bytes(c) + proj_workspace_bytes(C, C, 3) + proj_workspace_bytes(C, C, 1);
+    const size_t total = 4 * block_tensor_bytes(c);
     if (cudaMalloc(&c->block_ws, total) != cudaSuccess) {
         cudaGetLastError();
         c->block_ws = nullptr;
@@ -396,11 +406,10 @@ slide_attn_status slide_attn_project(slide_attn_ctx* c, const void* x, const flo
         if (y[i] == x) return SLIDE_ATTN_ERR_INVALID_ARG;
         for (int j = 0; j < i; ++j) if (y[i] == y[j]) return SLIDE_ATTN_ERR_INVALID_ARG;
     }
-    slide_attn_status st = block_scratch(c);
+    slide_attn_status st = proj_check(c);
     if (st != SLIDE_ATTN_OK) return st;
     const int C = c->heads * c->head_dim;
-    unsigned char* img = static_cast<unsigned char*>(c->block_ws) + 4 * block_tensor_bytes(c);
-    if (launch_proj(x, (long long)c->B * c->H * c->W, C, w, C, nmat, y, img, c->d_status, c->num_sms,
+    if (launch_proj(x, (long long)c->B * c->H * c->W, C, w, C, nmat, y, c->d_status, c->num_sms,
                     static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
         cudaGetLastError();
         return SLIDE_ATTN_ERR_CUDA;
@@ -428,10 +437,8 @@ slide_attn_status slide_attn_block_forward(slide_attn_ctx* c, const void* x, con
     unsigned char* base = static_cast<unsigned char*>(c->block_ws);
     void* qkv[3] = {base, base + tb, base + 2 * tb};
     void* z = base + 3 * tb;
-    unsigned char* img_qkv = base + 4 * tb;
-    unsigned char* img_o = img_qkv + proj_workspace_bytes(C, C, 3);
 
-    if (launch_proj(x, rows, C, w_qkv, C, 3, qkv, img_qkv, c->d_status, c->num_sms, stream) != cudaSuccess) {
+    if (launch_proj(x, rows, C, w_qkv, C, 3, qkv, c->d_status, c->num_sms, stream) != cudaSuccess) {
         cudaGetLastError();
         return SLIDE_ATTN_ERR_CUDA;
     }
@@ -442,7 +449,7 @@ slide_attn_status slide_attn_block_forward(slide_attn_ctx* c, const void* x, con
     st = launch_problem(c, p, stream, false);
     if (st != SLIDE_ATTN_OK) return st;
     void* ys[1] = {out};
-    if (launch_proj(z, rows, C, w_o, C, 1, ys, img_o, c->d_status, c->num_sms, stream) != cudaSuccess) {
+    if (launch_proj(z, rows, C, w_o, C, 1, ys, c->d_status, c->num_sms, stream) != cudaSuccess) {
         cudaGetLastError();
         return SLIDE_ATTN_ERR_CUDA;
     }

@@ -12,10 +12,11 @@
 //   X tile   [K/8][128 rows][16 B]   written by K/8 TMA boxes of 8 channels x 128 rows (rows past the end read 0)
 //   W chunk  [K/8][nch cols][16 B]   built from the fp32 weights by the epilogue warps while the first X tiles load
 //
-// Warps: 0 TMA producer, 1 MMA issuer (owns tensor memory), 2-9 epilogue (TMEM lane quarter = warp % 4, two warps
-// per quarter taking the column passes in turn: one thread per accumulator row, tcgen05.ld.32x32b -> bf16 -> a padded staging patch in shared memory -> row-major
-// 16-byte stores of whole sectors).  Two accumulator slots of 256 columns let
-// the MMAs of item i+1 run under the epilogue of item i.  Every wait is bounded; a wait that runs out sets the
+// Warps: 0 TMA producer, 1 MMA issuer (owns tensor memory), 2-17 epilogue in four groups of four (TMEM lane quarter
+// = warp % 4; a group owns every fourth work item, because one item's epilogue is a chain of dependent latencies of
+// about 850 cycles: one thread per accumulator row, tcgen05.ld.32x32b -> bf16 -> a padded staging patch in shared
+// memory -> row-major 16-byte stores of whole sectors).  Tensor memory holds 512 / nch accumulator slots (at most
+// eight), so the MMAs run ahead of the epilogue.  Every wait is bounded; a wait that runs out sets the
 // status word and the kernel still releases tensor memory.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -24,19 +25,20 @@ namespace slide_attn {
 
 namespace {
 
-constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter: they take the column passes of an item in turn
+constexpr int kGroups = 4;                   // epilogue warp groups; group g owns the items it = g (mod kGroups)
+constexpr int kEpiWarps = 4 * kGroups;       // one warp per TMEM lane quarter in every group
 constexpr int kThreads = (2 + kEpiWarps) * 32;
 constexpr int kMaxStages = 6;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kSlotCols = 256;
+constexpr int kMaxSlots = 8;                 // accumulator slots in tensor memory: 512 / nch, at most this many
 constexpr size_t kMaxSmem = 227 * 1024;
 
 constexpr int kBarXFull = 0;                 // [kMaxStages]
 constexpr int kBarXEmpty = kMaxStages;       // [kMaxStages]  one arrival: the commit behind the tile's last MMA
 constexpr int kBarWeights = 2 * kMaxStages;  // count kEpiWarps: the weight images are in shared memory
-constexpr int kBarAccFull = kBarWeights + 1; // [2]
-constexpr int kBarAccFree = kBarAccFull + 2; // [2]  count kEpiWarps
-constexpr int kNumBars = kBarAccFree + 2;
+constexpr int kBarAccFull = kBarWeights + 1; // [kMaxSlots]
+constexpr int kBarAccFree = kBarAccFull + kMaxSlots; // [kMaxSlots]  count 4: the four warps of the group that owned the item
+constexpr int kNumBars = kBarAccFree + kMaxSlots;
 
 struct ProjParams {
     const float* w;              // nmat row-major [K][ycols] matrices, one after the other
@@ -112,11 +114,12 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
     const int ntiles = (P.rows + 127) >> 7;
     const int my_tiles = (int)blockIdx.x < ntiles ? (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     const int S = P.stages;
+    const int nslots = 512 / P.nch < kMaxSlots ? 512 / P.nch : kMaxSlots;      // >= 2: nch <= 256
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init_only(bar(kBarXFull + s), 1); mbar_init_only(bar(kBarXEmpty + s), 1); }
         mbar_init_only(bar(kBarWeights), kEpiWarps);
-        for (int i = 0; i < 2; ++i) { mbar_init_only(bar(kBarAccFull + i), 1); mbar_init_only(bar(kBarAccFree + i), kEpiWarps); }
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init_only(bar(kBarAccFull + i), 1); mbar_init_only(bar(kBarAccFree + i), 4); }
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(smem + tmem_off), kTmemCols);
@@ -132,12 +135,13 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
         uint32_t leader;
         if (elect_one(leader) && my_tiles > 0) {
             grid_dependency_wait();
-            for (int t = 0; ok && t < my_tiles; ++t) {
-                const int s = t % S, m = (int)blockIdx.x + t * (int)gridDim.x;
-                if (!mbar_wait(bar(kBarXEmpty + s), (uint32_t)(((t / S) & 1) ^ 1))) { ok = false; break; }
+            int s = 0, phase = 0;                                // stage t % S and the parity of its t / S-th use
+            for (int t = 0, m = (int)blockIdx.x; ok && t < my_tiles; ++t, m += (int)gridDim.x) {
+                if (!mbar_wait(bar(kBarXEmpty + s), (uint32_t)(phase ^ 1))) { ok = false; break; }
                 const uint32_t dst = smem_u32(smem + x_off + (size_t)s * stage_bytes), fb = bar(kBarXFull + s);
                 mbar_expect_tx(fb, stage_bytes);
                 for (int kg = 0; kg < (P.K >> 3); ++kg) tma_load_4d(dst + (uint32_t)kg * 2048u, &map_x, fb, 8 * kg, m * 128, 0, 0);
+                if (++s == S) { s = 0; phase ^= 1; }
             }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
@@ -150,23 +154,24 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
             const uint32_t b_lbo = (uint32_t)P.nch * 16u;
             const uint32_t sB0 = smem_u32(smem);
             if (!mbar_wait(bar(kBarWeights), 0)) ok = false;
-            int it = 0;
+            int s = 0, phase = 0, slot = 0, slot_phase = 0;
             for (int t = 0; ok && t < my_tiles; ++t) {
-                const int s = t % S;
-                if (!mbar_wait(bar(kBarXFull + s), (uint32_t)((t / S) & 1))) { ok = false; break; }
-                const uint32_t sX = smem_u32(smem + x_off + (size_t)s * stage_bytes);
-                for (int ch = 0; ch < P.nchunks; ++ch, ++it) {
-                    const int slot = it & 1;
-                    if (!mbar_wait(bar(kBarAccFree + slot), (uint32_t)(((it >> 1) & 1) ^ 1))) { ok = false; break; }
+                if (!mbar_wait(bar(kBarXFull + s), (uint32_t)phase)) { ok = false; break; }
+                // descriptors step in 16-byte units: two planes of X and two K-groups of the chunk per MMA
+                const uint64_t adesc0 = umma_smem_desc(smem_u32(smem + x_off + (size_t)s * stage_bytes), 2048, 128);
+                uint64_t bdesc0 = umma_smem_desc(sB0, b_lbo, 128);
+                for (int ch = 0; ch < P.nchunks; ++ch, bdesc0 += chunk_bytes >> 4) {
+                    if (!mbar_wait(bar(kBarAccFree + slot), (uint32_t)(slot_phase ^ 1))) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t dcol = tmem + (uint32_t)slot * kSlotCols;
-                    const uint32_t sB = sB0 + (uint32_t)ch * chunk_bytes;
-                    for (int kk = 0; kk < (P.K >> 4); ++kk)
-                        umma_bf16_ss(dcol, umma_smem_desc(sX + (uint32_t)kk * 4096u, 2048, 128),
-                                     umma_smem_desc(sB + (uint32_t)kk * 2u * b_lbo, b_lbo, 128), idesc, kk > 0 ? 1u : 0u);
+                    const uint32_t dcol = tmem + (uint32_t)(slot * P.nch);
+                    uint64_t adesc = adesc0, bdesc = bdesc0;
+                    for (int kk = 0; kk < (P.K >> 4); ++kk, adesc += 4096u >> 4, bdesc += (2u * b_lbo) >> 4)
+                        umma_bf16_ss(dcol, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
                     umma_commit(bar(kBarAccFull + slot));
+                    if (++slot == nslots) { slot = 0; slot_phase ^= 1; }
                 }
                 if (ok) umma_commit(bar(kBarXEmpty + s));       // the tile's last MMA has read it
+                if (++s == S) { s = 0; phase ^= 1; }
             }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, leader) != 0;
@@ -175,7 +180,7 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
         // the lane's row goes TMEM -> registers -> bf16 -> a staging row of this warp in shared memory (row pitch
         // 2 SW + 16 bytes: conflict-free 16-byte stores), then the warp writes the 32 x SW patch to global memory in
         // row-major order, 16 bytes per lane, so that every row segment leaves as whole 32-byte sectors.
-        const int sub = warp & 3, half = (warp - 2) >> 2;
+        const int sub = warp & 3, group = (warp - 2) >> 2;
         const uint32_t tlane = tmem + ((uint32_t)(32 * sub) << 16);
         unsigned char* stg = smem + stage_off + (size_t)(warp - 2) * (size_t)(32 * (P.sw_max * 2 + 16));
         if (my_tiles > 0) {
@@ -199,30 +204,39 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarWeights));
         }
-        int it = 0;
+        // items in launch order: it = t * nchunks + ch.  This warp's group owns the items it = group (mod ngroups): it
+        // waits for, reads and releases only those; for the others it merely advances the slot and column counters.
+        // No more groups take part than there are slots: a group then always waits on a phase of a slot's barrier whose
+        // predecessor it knows to be complete (its previous item came later than this slot's previous use), so the
+        // parity test cannot be satisfied by an older phase.
+        const int ngroups = nslots < kGroups ? nslots : kGroups;
+        const int t0 = P.n0 / P.ycols, c00 = P.n0 - t0 * P.ycols;     // tensor and column of the launch's first chunk
+        int slot = 0, slot_phase = 0, turn = 0;                       // turn = it mod ngroups
         for (int t = 0; ok && t < my_tiles; ++t) {
             const long long row0 = ((long long)blockIdx.x + (long long)t * gridDim.x) * 128 + 32 * sub;
             const int rows_left = (long long)P.rows - row0 > 32 ? 32 : (int)((long long)P.rows - row0);   // may be <= 0
-            for (int ch = 0; ch < P.nchunks; ++ch, ++it) {
-                const int slot = it & 1;
-                if (!warp_wait(bar(kBarAccFull + slot), (uint32_t)((it >> 1) & 1))) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t tacc = tlane + (uint32_t)slot * kSlotCols;
-                int c = 0;
-                for (int pass = 0; c < P.nch; ++pass) {
-                    const int sw = (P.nch - c >= 64 && P.sw_max >= 64) ? 64 : (P.nch - c >= 32 ? 32 : 16);
-                    if (((pass + it) & 1) != half) { c += sw; continue; }
-                    const int n = P.n0 + ch * P.nch + c;                 // a pass never straddles two tensors
-                    const int ti = n / P.ycols, col = n - ti * P.ycols;
-                    __nv_bfloat16* ybase = P.y[ti] + (size_t)row0 * P.ycols + col;
-                    if (sw == 64) store_cols<64>(tacc + (uint32_t)c, stg, lane, ybase, P.ycols, rows_left);
-                    else if (sw == 32) store_cols<32>(tacc + (uint32_t)c, stg, lane, ybase, P.ycols, rows_left);
-                    else store_cols<16>(tacc + (uint32_t)c, stg, lane, ybase, P.ycols, rows_left);
-                    c += sw;
+            int ti = t0, col0 = c00;                                  // a chunk lies within one tensor
+            for (int ch = 0; ch < P.nchunks; ++ch) {
+                if (turn == group) {
+                    if (!warp_wait(bar(kBarAccFull + slot), (uint32_t)slot_phase)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t tacc = tlane + (uint32_t)(slot * P.nch);
+                    __nv_bfloat16* ybase = P.y[ti] + (size_t)row0 * P.ycols + col0;
+                    for (int c = 0; c < P.nch;) {
+                        const int sw = (P.nch - c >= 64 && P.sw_max >= 64) ? 64 : (P.nch - c >= 32 ? 32 : 16);
+                        if (sw == 64) store_cols<64>(tacc + (uint32_t)c, stg, lane, ybase + c, P.ycols, rows_left);
+                        else if (sw == 32) store_cols<32>(tacc + (uint32_t)c, stg, lane, ybase + c, P.ycols, rows_left);
+                        else store_cols<16>(tacc + (uint32_t)c, stg, lane, ybase + c, P.ycols, rows_left);
+                        c += sw;
+                    }
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarAccFree + slot));
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarAccFree + slot));
+                if (++turn == ngroups) turn = 0;
+                if (++slot == nslots) { slot = 0; slot_phase ^= 1; }
+                col0 += P.nch;
+                if (col0 == P.ycols) { col0 = 0; ++ti; }
             }
         }
     }

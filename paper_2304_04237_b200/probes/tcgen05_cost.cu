@@ -3,7 +3,7 @@
 //   1. back-to-back tcgen05.mma (M = 128, K = 16, bf16 -> fp32), fully unrolled so that the issuing
 //      thread executes nothing else: cycles per instruction as a function of N, of the A operand's
 //      home (shared memory / tensor memory), of the number of accumulator tiles the sequence
-//      alternates between and of the number of issuing threads; and the latency from the last issue
+//      alternates between, of the shared-memory layout of the operands and of the number of issuing threads; and the latency from the last issue
 //      to the wake-up of a thread waiting on the commit barrier
 //   2. tensor-memory loads and stores (issue -> wait complete) for one warp
 //   3. a wait on an mbarrier phase that is already complete, in the forms the kernels could use, each
@@ -49,15 +49,17 @@ __global__ void __launch_bounds__(192, 1) mma_seq(Res* res)
         uint32_t leader;
         if (elect_one(leader)) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, N);
-            const uint64_t adesc = umma_smem_desc(smem_u32(sA), 128, 256);
-            const uint64_t bdesc = umma_smem_desc(smem_u32(sB), 128, 256);
+            // MODE 0: the two K-halves of an 8-row group lie side by side (LBO 128, SBO 256);
+            // MODE 2: K-halves as separate planes of all rows (A: LBO 2048, SBO 128; B: LBO 16 N, SBO 128)
+            const uint64_t adesc = MODE == 2 ? umma_smem_desc(smem_u32(sA), 2048, 128) : umma_smem_desc(smem_u32(sA), 128, 256);
+            const uint64_t bdesc = MODE == 2 ? umma_smem_desc(smem_u32(sB), 16 * N, 128) : umma_smem_desc(smem_u32(sB), 128, 256);
             const uint32_t acol = tmem + 504;        // A operand of the .ts form: 8 columns
             const uint32_t bar = smem_u32(&bars[me]);
             const uint32_t d0 = tmem + (uint32_t)(me * NT * N);
             const long long t0 = clock64();
 #pragma unroll
             for (int i = 0; i < COUNT; ++i) {
-                if (MODE == 0) umma_bf16_ss(d0 + (uint32_t)((i % NT) * N), adesc, bdesc, idesc, i >= NT ? 1u : 0u);
+                if (MODE != 1) umma_bf16_ss(d0 + (uint32_t)((i % NT) * N), adesc, bdesc, idesc, i >= NT ? 1u : 0u);
                 else umma_bf16_ts(d0 + (uint32_t)((i % NT) * N), acol, bdesc, idesc, i >= NT ? 1u : 0u);
             }
             const long long t1 = clock64();
@@ -210,7 +212,7 @@ void run(Res* d)
     }
     CK(cudaMemcpy(h, d, sizeof(h), cudaMemcpyDeviceToHost));
     for (int me = 0; me < ISSUERS; ++me)
-        printf("| %s | %3d | %d | %3d | %d | %6lld | %6lld | %6.1f | %6lld | %d |\n", MODE ? "tensor memory" : "shared memory", N, NT, COUNT,
+        printf("| %s | %3d | %d | %3d | %d | %6lld | %6lld | %6.1f | %6lld | %d |\n", MODE == 1 ? "tensor memory" : MODE == 2 ? "shared memory, K-halves as planes" : "shared memory", N, NT, COUNT,
                ISSUERS, h[me].issue, h[me].total, (double)h[me].issue / COUNT, h[me].total - h[me].issue, h[me].ok);
 }
 
@@ -222,7 +224,8 @@ int main()
     run<1, 64, 1, 72, 1>(d);  run<1, 64, 2, 72, 1>(d);  run<1, 96, 1, 72, 1>(d);  run<1, 96, 2, 72, 1>(d);  run<1, 112, 1, 72, 1>(d);
     run<1, 128, 1, 72, 1>(d); run<1, 256, 1, 72, 1>(d);
     run<0, 32, 1, 72, 1>(d);  run<0, 32, 2, 72, 1>(d);  run<0, 64, 1, 72, 1>(d);  run<0, 96, 1, 72, 1>(d);
-    run<0, 128, 1, 72, 1>(d); run<0, 256, 1, 72, 1>(d);
+    run<0, 128, 1, 72, 1>(d); run<0, 192, 1, 72, 1>(d); run<0, 256, 1, 72, 1>(d);
+    run<2, 32, 1, 72, 1>(d);  run<2, 64, 1, 72, 1>(d);  run<2, 128, 1, 72, 1>(d); run<2, 192, 1, 72, 1>(d); run<2, 256, 1, 72, 1>(d);
     run<1, 32, 1, 72, 2>(d);  run<1, 96, 1, 72, 2>(d);  run<0, 32, 1, 72, 2>(d);
     run<1, 32, 1, 3, 1>(d);   run<1, 96, 1, 2, 1>(d);
 

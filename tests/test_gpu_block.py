@@ -65,7 +65,10 @@ def test_project_is_bit_exact_on_small_integers(shape, nmat):
         np.testing.assert_array_equal(got[m], want)
 
 
-@pytest.mark.parametrize("shape", [(2, 14, 14, 64), (1, 33, 47, 96), (1, 28, 28, 192), (1, 20, 20, 256)], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("shape", [(2, 14, 14, 64), (1, 33, 47, 96), (1, 28, 28, 192), (1, 20, 20, 256),
+                                   # more than two row tiles per CTA, for every number of accumulator slots
+                                   (1, 210, 200, 32), (1, 200, 200, 96), (1, 200, 200, 128), (1, 200, 200, 192), (1, 199, 200, 256)],
+                         ids=lambda s: "x".join(map(str, s)))
 def test_project_random_matches_double(shape):
     B, H, W, C = shape
     rng = np.random.default_rng(zlib.crc32(repr(shape).encode()))

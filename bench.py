@@ -307,11 +307,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other", action="store_true", help="skip the kernel-only figures of the other gated shapes")
-    ap.add_argument("--backward", type=int, default=0, metavar="N",
-                    help="also time N backward passes (slide_attn_backward) of the workload and report them beside the forward")
-    ap.add_argument("--block", type=int, default=0, metavar="N",
+    ap.add_argument("--backward", type=int, default=20, metavar="N",
+                    help="also time N backward passes (slide_attn_backward) of the workload and report them beside the forward "
+                         "(single-GPU runs, window sizes the backward supports; 0 = off)")
+    ap.add_argument("--block", type=int, default=200, metavar="N",
                     help="also time N whole blocks (slide_attn_block_forward: Eq. 1 projections, attention, Eq. 3 projection) "
-                         "on the workload's shape and report them beside the forward")
+                         "on the workload's shape and report them beside the forward (single-GPU runs, bf16; 0 = off)")
     ap.add_argument("--fixed-shift", action="store_true",
                     help="the workload with exactly one-hot depthwise weights (sigma_w = 0), run in fixed-shift mode")
     args = ap.parse_args()
@@ -417,7 +418,7 @@ def main():
 
     # optional: the backward pass of the same workload (gradients of all six inputs)
     backward = None
-    if args.backward > 0:
+    if args.backward > 0 and world == 1 and cfg["ksize"] <= 3 and cfg["head_dim"] == 32:
         s0 = sets[0]
         g = torch.randn_like(s0["q"])
         dq, dk, dv = (torch.empty_like(s0["q"]) for _ in range(3))
@@ -440,7 +441,7 @@ def main():
 
     # optional: a whole block on the workload's shape (projections on tcgen05 around the attention stage)
     block = None
-    if args.block > 0 and cfg["dtype"] == "bf16":
+    if args.block > 0 and world == 1 and cfg["dtype"] == "bf16":
         C = cfg["heads"] * cfg["head_dim"]
         gen = torch.Generator(device="cuda").manual_seed(1234)
         xs = [torch.randn((cfg["B"], cfg["H"], cfg["W"], C), device="cuda", generator=gen).to(torch.bfloat16) for _ in range(2)]

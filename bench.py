@@ -437,7 +437,7 @@ def main():
         assert sa.slide_attn_query_status(ctx) == sa.OK
         bms = a.elapsed_time(b) / args.backward
         backward = {"ms_per_step": bms, "steps": args.backward, "value": npx / (bms * 1e-3), "unit": UNIT,
-                    "kernels": "weight transpose, point kernel (a, dl, dq, dW, dbias), gather kernel (dk, dv)"}
+                    "kernels": "weight transpose, point kernel (a, dl, dq, dbias), gather kernel (dk, dv), weight kernel (dWk, dWv)"}
 
     # optional: a whole block on the workload's shape (projections on tcgen05 around the attention stage)
     block = None
@@ -471,7 +471,7 @@ def main():
                  "proj_qkv_ms": qkv_ms, "proj_qkv_gbs": 4 * tok_bytes / (qkv_ms * 1e-3) / 1e9,
                  "proj_o_ms": o_ms, "proj_o_gbs": 2 * tok_bytes / (o_ms * 1e-3) / 1e9,
                  "bytes_min_three_stages": 10 * tok_bytes, "bytes_min_fused": 2 * tok_bytes,
-                 "kernels": "weight images + projection GEMM (Eq. 1), attention, weight image + projection GEMM (Eq. 3)"}
+                 "kernels": "projection GEMM (Eq. 1, three outputs), attention (prep + main), projection GEMM (Eq. 3)"}
 
     # end to end through the host-buffer entry point: pinned host inputs in, pinned result out
     e2e = None

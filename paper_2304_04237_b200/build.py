@@ -1,6 +1,6 @@
 """Builds libslide_attn.so (sm_100a) from csrc/ with nvcc, in-tree.
 
-    python -m paper_2304_04237_b200.build [--force] [--verbose]
+    python -m paper_2304_04237_b200.build [--force] [--verbose] [--probes] [--timeline]
 
 Objects go to paper_2304_04237_b200/_build/, the library next to this file.  nvcc
 cross-compiles, so no GPU is needed to build.
@@ -85,7 +85,31 @@ def build_probes() -> list:
     return outs
 
 
+def build_timeline() -> str:
+    """A second copy of the library with -DSLIDE_ATTN_TIMELINE (clock stamps in the projection kernel's role loops),
+    as probes/_build/libslide_attn_timeline.so; read by probes/proj_timeline.py."""
+    out_dir = os.path.join(HERE, "probes", "_build", "timeline")
+    os.makedirs(out_dir, exist_ok=True)
+    objs = []
+    for s in sorted(glob.glob(os.path.join(CSRC, "*.cu"))):
+        o = os.path.join(out_dir, os.path.basename(s)[:-3] + ".o")
+        r = subprocess.run([_nvcc(), *NVCC_FLAGS, "-DSLIDE_ATTN_TIMELINE", "-c", s, "-o", o], capture_output=True, text=True)
+        if r.returncode != 0:
+            sys.stderr.write(r.stdout + r.stderr)
+            raise RuntimeError("nvcc failed for " + s)
+        objs.append(o)
+    lib = os.path.join(HERE, "probes", "_build", "libslide_attn_timeline.so")
+    r = subprocess.run([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", *objs, "-o", lib],
+                       capture_output=True, text=True)
+    if r.returncode != 0:
+        sys.stderr.write(r.stdout + r.stderr)
+        raise RuntimeError("link failed")
+    return lib
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
     if "--probes" in sys.argv:
         print("\n".join(build_probes()))
+    if "--timeline" in sys.argv:
+        print(build_timeline())

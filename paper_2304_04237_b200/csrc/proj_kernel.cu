@@ -11,6 +11,10 @@
 // Shared-memory operand layout (no swizzle, K-major core matrices of 8 rows x 16 bytes):
 //   X tile   [K/8][128 rows][16 B]   written by K/8 TMA boxes of 8 channels x 128 rows (rows past the end read 0)
 //   W chunk  [K/8][nch cols][16 B]   built from the fp32 weights by the epilogue warps while the first X tiles load
+// The X boxes fetch a 32-byte sector for every 16 bytes, and with the three output tensors that L2 traffic is what
+// bounds the kernel.  Measured and not kept: four producer warps copying the tile with cp.async in row-major order
+// of the source (whole lines; planes padded by 16 bytes against bank conflicts; one or two free stages beyond the
+// tiles in flight) - 32.5 / 18.0 us for the two projections of a 64-channel block against 21.1 / 12.7 with the boxes.
 //
 // Warps: 0 TMA producer, 1 MMA issuer (owns tensor memory), 2-17 epilogue in four groups of four (TMEM lane quarter
 // = warp % 4; a group owns every fourth work item, because one item's epilogue is a chain of dependent latencies of
@@ -22,6 +26,16 @@
 #include "ptx.cuh"
 
 namespace slide_attn {
+
+// Time-line build (-DSLIDE_ATTN_TIMELINE, `python -m paper_2304_04237_b200.build --timeline`): CTA 0 stamps clock64
+// at six points of its role loops, per work item; slide_attn_proj_timeline copies the stamps out.  The stamps cost a
+// few instructions and skip no work; the library proper is built without them.
+#ifdef SLIDE_ATTN_TIMELINE
+__device__ long long g_proj_timeline[6][256];
+#define PROJ_TL(role, idx) do { if (blockIdx.x == 0 && (idx) < 256) g_proj_timeline[role][idx] = clock64(); } while (0)
+#else
+#define PROJ_TL(role, idx) do {} while (0)
+#endif
 
 namespace {
 
@@ -154,20 +168,23 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
             const uint32_t b_lbo = (uint32_t)P.nch * 16u;
             const uint32_t sB0 = smem_u32(smem);
             if (!mbar_wait(bar(kBarWeights), 0)) ok = false;
-            int s = 0, phase = 0, slot = 0, slot_phase = 0;
+            int s = 0, phase = 0, slot = 0, slot_phase = 0, it = 0;
             for (int t = 0; ok && t < my_tiles; ++t) {
                 if (!mbar_wait(bar(kBarXFull + s), (uint32_t)phase)) { ok = false; break; }
                 // descriptors step in 16-byte units: two planes of X and two K-groups of the chunk per MMA
                 const uint64_t adesc0 = umma_smem_desc(smem_u32(smem + x_off + (size_t)s * stage_bytes), 2048, 128);
                 uint64_t bdesc0 = umma_smem_desc(sB0, b_lbo, 128);
-                for (int ch = 0; ch < P.nchunks; ++ch, bdesc0 += chunk_bytes >> 4) {
+                for (int ch = 0; ch < P.nchunks; ++ch, ++it, bdesc0 += chunk_bytes >> 4) {
+                    PROJ_TL(0, it);                              // MMA thread turns to the item
                     if (!mbar_wait(bar(kBarAccFree + slot), (uint32_t)(slot_phase ^ 1))) { ok = false; break; }
+                    PROJ_TL(1, it);                              // its accumulator slot is free
                     tc_fence_after_sync();
                     const uint32_t dcol = tmem + (uint32_t)(slot * P.nch);
                     uint64_t adesc = adesc0, bdesc = bdesc0;
                     for (int kk = 0; kk < (P.K >> 4); ++kk, adesc += 4096u >> 4, bdesc += (2u * b_lbo) >> 4)
                         umma_bf16_ss(dcol, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
                     umma_commit(bar(kBarAccFull + slot));
+                    PROJ_TL(2, it);                              // MMAs and commit issued
                     if (++slot == nslots) { slot = 0; slot_phase ^= 1; }
                 }
                 if (ok) umma_commit(bar(kBarXEmpty + s));       // the tile's last MMA has read it
@@ -211,14 +228,16 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
         // parity test cannot be satisfied by an older phase.
         const int ngroups = nslots < kGroups ? nslots : kGroups;
         const int t0 = P.n0 / P.ycols, c00 = P.n0 - t0 * P.ycols;     // tensor and column of the launch's first chunk
-        int slot = 0, slot_phase = 0, turn = 0;                       // turn = it mod ngroups
+        int slot = 0, slot_phase = 0, turn = 0, it = 0;               // turn = it mod ngroups
         for (int t = 0; ok && t < my_tiles; ++t) {
             const long long row0 = ((long long)blockIdx.x + (long long)t * gridDim.x) * 128 + 32 * sub;
             const int rows_left = (long long)P.rows - row0 > 32 ? 32 : (int)((long long)P.rows - row0);   // may be <= 0
             int ti = t0, col0 = c00;                                  // a chunk lies within one tensor
-            for (int ch = 0; ch < P.nchunks; ++ch) {
+            for (int ch = 0; ch < P.nchunks; ++ch, ++it) {
                 if (turn == group) {
+                    if (sub == 0 && lane == 0) PROJ_TL(3, it);   // the owning group's first warp turns to the item
                     if (!warp_wait(bar(kBarAccFull + slot), (uint32_t)slot_phase)) { ok = false; break; }
+                    if (sub == 0 && lane == 0) PROJ_TL(4, it);   // accumulator seen
                     tc_fence_after_sync();
                     const uint32_t tacc = tlane + (uint32_t)(slot * P.nch);
                     __nv_bfloat16* ybase = P.y[ti] + (size_t)row0 * P.ycols + col0;
@@ -229,6 +248,7 @@ proj_kernel(const __grid_constant__ CUtensorMap map_x, const ProjParams P)
                         else store_cols<16>(tacc + (uint32_t)c, stg, lane, ybase + c, P.ycols, rows_left);
                         c += sw;
                     }
+                    if (sub == 0 && lane == 0) PROJ_TL(5, it);   // stored; about to release the slot
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarAccFree + slot));
@@ -335,3 +355,10 @@ cudaError_t launch_proj(const void* x, long long rows, int c_in, const float* w,
 }
 
 }  // namespace slide_attn
+
+#ifdef SLIDE_ATTN_TIMELINE
+// host [6][256]: per work item of CTA 0 the clock64 stamps listed at PROJ_TL; returns the cudaError_t of the copy
+extern "C" int slide_attn_proj_timeline(long long* host) {
+    return (int)cudaMemcpyFromSymbol(host, slide_attn::g_proj_timeline, sizeof(long long) * 6 * 256);
+}
+#endif

@@ -6,11 +6,11 @@
 //   product warps   P[p,(t,c)] = q[p,c] k[p+off(t),c]   packed bf16 multiply -> tcgen05.st (TMEM)
 //   key MMA         L[p,n]     = sum_{t,c} P[p,(t,c)] Bk[(t,c),n]       tcgen05.mma, A from TMEM
 //                   n = 0..8: deformed part D_k of slot n;  n = 9..17: plain q.k sum of tap n-9
-//   product warps   logit[s] = (L[s] + L[9+s]) scale + bias[s];  e = exp2(logit - max)
+//   product warps   logit[s] = (L[s] + L[9+s]) scale + bias[s];  e = exp2(logit - max) / sum_s exp2(logit - max)
 //                   (tcgen05.ld.32x32b: one thread holds all logits of one pixel, no shuffles)
 //                   A' row = e_hi | e_hi | e_lo | e8_hi e8_hi e8_lo 0..   -> tcgen05.st (TMEM)
-//   value MMA       D[p,(t,c)] = sum_k A'[p,k] Bv[k,(t,c)]  (+16 sum columns)   A from TMEM
-//   value warps     out[p,c] = (sum_t D[p,t,c] v[p+off(t),c]) / sum[p]
+//   value MMA       D[p,(t,c)] = sum_k A'[p,k] Bv[k,(t,c)]                     A from TMEM
+//   value warps     out[p,c] = sum_t D[p,t,c] v[p+off(t),c]
 //
 // Tensor memory (512 columns): two value-chunk slots of 112 (chunk c = 3 blk + dx -> slot c & 1), four
 // P chunks of 48 (3 taps x 32 bf16, chunk -> buffer c & 3), two logit tiles of 32, two A' tiles of 16.
@@ -46,7 +46,7 @@ constexpr int kCtlT = kCtlK2 + 1;                       // warp 19: TMA thread, 
 constexpr int kThreads = (kCtlT + 1) * 32;
 constexpr int kKStages = 2;
 constexpr int kMaxVStages = 4;
-constexpr int kBCols = 304;                             // 288 value columns + 16 sum columns
+constexpr int kBCols = 288;                             // value columns: (tap, channel)
 constexpr int kBBytes = kBCols * 64;
 constexpr int kBkBytes = 36 * 512;                      // key-side B: 288 K x 32 N bf16
 constexpr int kImgBytes = kBBytes + kBkBytes;           // both B images of one head, as the prep kernel leaves them
@@ -58,7 +58,6 @@ constexpr uint32_t kColP = 224;                         // four P chunks of 48 c
 constexpr uint32_t kColL = 416;                         // two logit tiles of 32 columns
 constexpr uint32_t kColE = 480;                         // two A' tiles of 16 columns (32 bf16)
 constexpr uint32_t kIdesc96 = umma_idesc_bf16(128, 96);
-constexpr uint32_t kIdesc112 = umma_idesc_bf16(128, 112);
 constexpr uint32_t kIdesc32 = umma_idesc_bf16(128, 32);
 
 struct UmmaParams {
@@ -128,9 +127,9 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
 // Prep kernel: the two B images of every head, in the shared-memory layout the MMAs read
 // (K-major core matrices of 8 rows x 16 bytes, no swizzle), written to the context workspace once per
 // forward.  Block (h, part) builds a share of head h's items.
-//   value side  [304 columns][32 K] bf16: column n = (tap-column-major tap, channel); K rows
+//   value side  [288 columns][32 K] bf16: column n = (tap-column-major tap, channel); K rows
 //               0..7 D_v[c][s][t], 8..15 and 16..23 the one-hot [s = t], 24 D_v[c][8][t], 25, 26 [t = 8]
-//               (the A' row is e_hi | e_hi | e_lo | e8_hi e8_hi e8_lo); columns 288.. sum the A' row
+//               (the A' row is e_hi | e_hi | e_lo | e8_hi e8_hi e8_lo)
 //   key side    [288 K][32 N] bf16: K = 32 tap + kappa (kappa -> channel as tcgen05.st lays P out),
 //               N 0..8 D_k[c][n][t], 9..17 the one-hot [n - 9 = t]
 __global__ void __launch_bounds__(256)
@@ -149,11 +148,7 @@ umma_ts_prep_kernel(const float* __restrict__ wk, const float* __restrict__ wv, 
             uint32_t w[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) w[i] = 0u;
-            if (n >= 288) {
-#pragma unroll
-                for (int i = 4; i < 12; ++i) w[i] = kOnesBf16x2;
-                w[12] = pack_bf16(0.f, 1.f); w[13] = pack_bf16(1.f, 0.f);
-            } else {
+            {
                 const int ts = n >> 5, t = (ts % 3) * 3 + ts / 3;
                 const int cn = n & 31, j = cn >> 3, wi = cn & 7;
                 const float* wc = wvs + (8 * (wi >> 1) + 2 * j + (wi & 1)) * 81 + t;
@@ -326,12 +321,16 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 float l[9], m = -INFINITY;
 #pragma unroll
                 for (int s = 0; s < 9; ++s) { l[s] = (Lg[s] + Lg[9 + s]) * P.scale_log2e + biasl[s]; m = fmaxf(m, l[s]); }
+                float e[9], sum = 0.f;
+#pragma unroll
+                for (int s = 0; s < 9; ++s) { e[s] = fast_exp2(l[s] - m); sum += e[s]; }
+                const float inv = rcp_approx(sum);               // the weights leave normalised: the value side only sums
                 float hi[9], lo[9];
 #pragma unroll
                 for (int s = 0; s < 9; ++s) {
-                    const float e = fast_exp2(l[s] - m);
-                    hi[s] = __bfloat162float(__float2bfloat16_rn(e));
-                    lo[s] = e - hi[s];
+                    const float a = e[s] * inv;
+                    hi[s] = __bfloat162float(__float2bfloat16_rn(a));
+                    lo[s] = a - hi[s];
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -441,7 +440,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             for (int i = 0; i < 2; ++i)
 #pragma unroll
                 for (int c = 0; c < 8; ++c) o_acc[i][c] = 0.f;
-            float inv[2] = {0.f, 0.f};
 
 #pragma unroll
             for (int dx = 0; dx < 3; ++dx) {
@@ -453,8 +451,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     uint32_t dr[48];
                     const uint32_t ta = tq + colbase;
                     tmem_ld3_16x256b_x4_nowait(ta, ta + 32, ta + 64, dr);
-                    uint32_t sr[4] = {0u, 0u, 0u, 0u};             // sum_s e[p,s] of the two pixels (last chunk)
-                    if (dx == 2) tmem_ld_16x256b_x1_nowait(tq + colbase + 96, sr);
                     uint4 vp[4];
 #pragma unroll
                     for (int r = 0; r < 4; ++r) vp[r] = lds_u4(sV, off0 + (uint32_t)((2 * m + r) * HW2 + dx) * 64u);
@@ -468,10 +464,6 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         vf[r][6] = bf16_lo(v.w); vf[r][7] = bf16_hi(v.w);
                     }
                     tmem_wait_ld48(dr);
-                    if (dx == 2) {
-                        tmem_pass4(sr);
-                        inv[0] = rcp_approx(__uint_as_float(sr[0])); inv[1] = rcp_approx(__uint_as_float(sr[2]));
-                    }
                     float d[48];
 #pragma unroll
                     for (int i = 0; i < 48; ++i) d[i] = __uint_as_float(dr[i]);
@@ -499,10 +491,10 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 for (int i = 0; i < 2; ++i) {
                     if (x < P.W && y0 + i < P.H) {
                         uint4 r;
-                        r.x = pack_bf16(o_acc[i][0] * inv[i], o_acc[i][1] * inv[i]);
-                        r.y = pack_bf16(o_acc[i][2] * inv[i], o_acc[i][3] * inv[i]);
-                        r.z = pack_bf16(o_acc[i][4] * inv[i], o_acc[i][5] * inv[i]);
-                        r.w = pack_bf16(o_acc[i][6] * inv[i], o_acc[i][7] * inv[i]);
+                        r.x = pack_bf16(o_acc[i][0], o_acc[i][1]);
+                        r.y = pack_bf16(o_acc[i][2], o_acc[i][3]);
+                        r.z = pack_bf16(o_acc[i][4], o_acc[i][5]);
+                        r.w = pack_bf16(o_acc[i][6], o_acc[i][7]);
                         *reinterpret_cast<uint4*>(op + i * row_stride) = r;
                     }
                 }
@@ -592,7 +584,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     if (!mbar_wait(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t sB = sB0 + dx * 12 * 512;
-                    const uint32_t idesc = dx == 2 ? kIdesc112 : kIdesc96;
+                    const uint32_t idesc = kIdesc96;
                     const uint32_t dcol = tmem + kColD + ds * 112;
                     umma_bf16_ts(dcol, acol, umma_smem_desc(sB, 128, 512), idesc, 0);
                     umma_bf16_ts(dcol, acol + 8, umma_smem_desc(sB + 256, 128, 512), idesc, 1);

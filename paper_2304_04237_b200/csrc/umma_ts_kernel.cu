@@ -34,6 +34,16 @@
 
 namespace slide_attn {
 
+// Time-line build (-DSLIDE_ATTN_TIMELINE): CTA 0 stamps clock64 around the waits of one warp of every role, per
+// chunk (c = 3 block + dx) or block; slide_attn_umma_ts_timeline copies the stamps out.  The stamps skip no work;
+// the library proper is built without them.
+#ifdef SLIDE_ATTN_TIMELINE
+__device__ long long g_umma_timeline[16][128];
+#define UMMA_TL(role, idx) do { if (blockIdx.x == 0 && (idx) < 128) g_umma_timeline[role][idx] = clock64(); } while (0)
+#else
+#define UMMA_TL(role, idx) do {} while (0)
+#endif
+
 namespace {
 
 constexpr int kHeadDim = 32;
@@ -308,7 +318,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // softmax of block sb (thread = pixel = TMEM lane 32 q + lane); `valid`: the unit exists
         auto softmax_block = [&](int sb, bool valid) -> bool {
             const int lb = sb & 1;
+            if (warp == kVWarps && lane == 0) UMMA_TL(3, sb);              // softmax of block sb: before the logits wait
             if (!warp_wait(bar(kBarLFull + lb), (sb >> 1) & 1)) return false;
+            if (warp == kVWarps && lane == 0) UMMA_TL(4, sb);
             tc_fence_after_sync();
             float Lg[32];
             tmem_ld_32x32b_x32(tq + kColL + 32 * lb, Lg);
@@ -341,7 +353,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 row[12] = pack_bf16(hi[8], hi[8]);
                 row[13] = pack_bf16(lo[8], 0.f);
             }
+            if (warp == kVWarps && lane == 0) UMMA_TL(5, sb);              // weights computed: before the A'-free wait
             if (!warp_wait(bar(kBarEFree + lb), ((sb >> 1) & 1) ^ 1)) return false;
+            if (warp == kVWarps && lane == 0) UMMA_TL(6, sb);
             tc_fence_after_sync();
             tmem_st_32x32b_x16(tq + kColE + 16 * lb, row);
             tmem_wait_st();
@@ -382,7 +396,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     uint4 kc[4];                                   // halo rows 2pm .. 2pm+3 of column dx
 #pragma unroll
                     for (int r = 0; r < 4; ++r) kc[r] = lds_u4(sK, off0 + (uint32_t)((2 * pm + r) * HW2 + dx) * 64u);
+                    if (warp == kVWarps && lane == 0) UMMA_TL(0, pc);      // product warp (0, 0): before the P-free wait
                     if (!warp_wait(bar(kBarPFree + pb), ((pc >> 2) & 1) ^ 1)) { ok = false; break; }
+                    if (warp == kVWarps && lane == 0) UMMA_TL(1, pc);      // after it
                     tc_fence_after_sync();
 #pragma unroll
                     for (int dy = 0; dy < 3; ++dy) {
@@ -397,6 +413,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     tmem_wait_st();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarPReady + pb));
+                    if (warp == kVWarps && lane == 0) UMMA_TL(2, pc);      // chunk delivered
                 }
                 if (!ok) break;
                 ++done_blocks;
@@ -444,7 +461,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
             for (int dx = 0; dx < 3; ++dx) {
                 const int cs = 3 * blk + dx, ds = cs & 1;
+                if (warp == 0 && lane == 0) UMMA_TL(7, cs);                // value warp (0, 0): before the chunk wait
                 if (!warp_wait(bar(kBarDFull + ds), (cs >> 1) & 1)) { ok = false; break; }
+                if (warp == 0 && lane == 0) UMMA_TL(8, cs);
                 tc_fence_after_sync();
                 const uint32_t colbase = kColD + ds * 112;
                 {
@@ -480,6 +499,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarDFree + ds));
+                if (warp == 0 && lane == 0) UMMA_TL(9, cs);                // chunk consumed
             }
             if (!ok) break;
 
@@ -540,7 +560,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
                 for (int dx = 0; dx < 3; ++dx) {
                     const int pc = 3 * blk + dx, pb = pc & 3;
+                    UMMA_TL(10, pc);                                       // key MMA thread: before the P-ready wait
                     if (!mbar_wait(bar(kBarPReady + pb), (pc >> 2) & 1)) { ok = false; break; }
+                    UMMA_TL(11, pc);
                     if (dx == 2) mbar_arrive(bar(kBarTurn + (me ^ 1)));
                     tc_fence_after_sync();
                     const uint32_t acol = tmem + kColP + 48 * pb;
@@ -553,6 +575,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                                          kIdesc32, (dx != 0 || dy != 0 || kh != 0) ? 1u : 0u);
                     }
                     umma_commit(bar(kBarPFree + pb));
+                    UMMA_TL(12, pc);                                       // MMAs and commit issued
                     if (dx == 2) umma_commit(bar(kBarLFull + lb));
                 }
             }
@@ -581,7 +604,9 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
                 for (int dx = 0; dx < 3; ++dx) {
                     const int cs = 3 * blk + dx, ds = cs & 1;
+                    UMMA_TL(13, cs);                                       // value MMA thread: before the slot-free wait
                     if (!mbar_wait(bar(kBarDFree + ds), ((cs >> 1) & 1) ^ 1)) { ok = false; break; }
+                    UMMA_TL(14, cs);
                     tc_fence_after_sync();
                     const uint32_t sB = sB0 + dx * 12 * 512;
                     const uint32_t idesc = kIdesc96;
@@ -589,6 +614,7 @@ umma_ts_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     umma_bf16_ts(dcol, acol, umma_smem_desc(sB, 128, 512), idesc, 0);
                     umma_bf16_ts(dcol, acol + 8, umma_smem_desc(sB + 256, 128, 512), idesc, 1);
                     umma_commit(bar(kBarDFull + ds));
+                    UMMA_TL(15, cs);
                     if (dx == 2) umma_commit(bar(kBarEFree + eb));
                 }
             }
@@ -716,3 +742,10 @@ cudaError_t launch_umma_ts(const Problem& p, const void* workspace, int* d_statu
 }
 
 }  // namespace slide_attn
+
+#ifdef SLIDE_ATTN_TIMELINE
+// host [16][128]: the clock64 stamps listed at UMMA_TL, indexed by chunk or block; returns the cudaError_t of the copy
+extern "C" int slide_attn_umma_ts_timeline(long long* host) {
+    return (int)cudaMemcpyFromSymbol(host, slide_attn::g_umma_timeline, sizeof(long long) * 16 * 128);
+}
+#endif

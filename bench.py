@@ -51,7 +51,7 @@ def algorithmic_bytes(cfg) -> int:
 NCU_TRAFFIC = {
     ("umma_ts", "c2"): {"bytes": 83.49e6,
                         "sources": ('paper_2304_04237_b200/csrc/umma_ts_kernel.cu', 'paper_2304_04237_b200/csrc/ptx.cuh'),
-                        "sha256": "ce86869dff783af87efc4bf23be2b9752cc227e5c2bd89bc6d42788559c5b3ce"},
+                        "sha256": "6c2f4e433aec8b8b57a0d6d1cc8f2be5a7dbd005c5f929bf5f1ac07841216743"},
     ("fixed_shift", "c2"): {"bytes": 85.38e6,
                             "sources": ('paper_2304_04237_b200/csrc/shift_kernel.cu', 'paper_2304_04237_b200/csrc/tile_common.cuh', 'paper_2304_04237_b200/csrc/ptx.cuh'),
                             "sha256": "d52af488501a9d58cb50407f1b82e038f60eae2056031d64999604761f99ad6c"},

@@ -12,10 +12,10 @@
 //   value MMA       D[p,(t,c)] = sum_k A'[p,k] Bv[k,(t,c)]                     A from TMEM
 //   value warps     out[p,c] = sum_t D[p,t,c] v[p+off(t),c]
 //
-// Tensor memory (512 columns): two value-chunk slots of 112 (chunk c = 3 blk + dx -> slot c & 1), four
-// P chunks of 48 (3 taps x 32 bf16, chunk -> buffer c & 3), two logit tiles of 32, two A' tiles of 16.
+// Tensor memory (512 columns): two value-chunk slots 112 columns apart, 96 used (chunk c = 3 blk + dx -> slot
+// c & 1), four P chunks of 48 (3 taps x 32 bf16, chunk -> buffer c & 3), two logit tiles of 32, two A' tiles of 16.
 //
-// Warps (20, 93 registers): 0-7 value warps (quadrant = warp % 4, pixel-row pair = warp / 4, every
+// Warps (20, 86 registers): 0-7 value warps (quadrant = warp % 4, pixel-row pair = warp / 4, every
 // block), 8-15 product warps (quadrant, pixel-row pair: P of their 16 pixels of every block; the
 // softmax of a block is done for the whole quadrant by the warp whose pair index equals the block's
 // parity, after it has stored the P of the next block), 16 and 18 key-side control (the 18 key MMAs
@@ -26,9 +26,10 @@
 // Warp 16 owns tensor memory.  Every wait is bounded; a wait that runs out sets the status word, and
 // tensor memory is released on every path.
 //
-// What bounds it: the tensor pipe takes about 85 cycles per MMA instruction however small
-// (18 of N = 32 and 6 of N = 96 / 112 per 128 pixels, 2.2 k cycles), the value warps need about as
-// long per block, and the measured block period is 2.9 k cycles.
+// What bounds it: instruction issue on the CUDA cores.  An M = 128 MMA costs about N / 2 cycles (18 of N = 32 and
+// 6 of N = 96 per 128 pixels: 540 cycles of a block period of about 2 850), the value warps are busy from block to
+// block, everything else waits for them, and with four or five warps per scheduler the time follows the instruction
+// count (5.9 k warp instructions per block: the q.k products, the widenings of V, the accumulator x V multiply-adds).
 #include "common.cuh"
 #include "ptx.cuh"
 
